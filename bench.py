@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the RaZeR matmul path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+
+One "step" is one pass of the decode hot path over one batch: the three Llama-7B-shaped
+GEMVs (M = 1; N x K = 4096x4096, 11008x4096, 4096x11008) against packed RaZeR weights.
+The headline value is the effective HBM bandwidth of that step: algorithmic bytes
+(N*K*0.5625 weight bytes + 2K activation + 2N output bytes per GEMV) over device time.
+Weights rotate over several distinct packed copies (> 500 MB in total, four times the L2)
+so every step streams from HBM.  Further lines of the same JSON object give the skinny
+(M = 4..64), prefill (M = 2048) and weight-activation results, the roofline fraction and
+the CPU oracle timed on the host cores.
+
+With --gpus N > 1 (launched by torchrun, one rank per GPU) every rank runs an independent
+replica of the same workload: the path has no exchange step, so there is no collective in
+the data path; the value is the sum over ranks over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+DECODE_SHAPES = [(4096, 4096), (11008, 4096), (4096, 11008)]
+SKINNY_SHAPES = [(8192, 8192), (28672, 8192), (8192, 28672)]
+PREFILL_SHAPES = [(14336, 4096), (4096, 14336)]
+METRIC = "razer_gemv_effective_hbm_bandwidth"
+
+
+def algo_bytes(M, N, K):
+    return N * K * 0.5625 + 2 * M * K + 2 * M * N
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                c = [v.strip() for v in ln.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); smax.append(float(c[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def time_cuda(fn, iters, torch):
+    """Device time of `iters` calls of fn(i), CUDA events on the current stream, ms per call."""
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for i in range(iters):
+        fn(i)
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / iters
+
+
+def make_sets(b, torch, inputs, N, K, n_sets, seed):
+    """n_sets distinct packed copies of an N x K random RaZeR tensor (rows rolled per copy)."""
+    codes, scales = inputs.random_codes(N, K, seed)
+    codes, scales = codes.cuda(), scales.cuda()
+    desc = b.make_desc(N, K, 0.002)
+    sets = []
+    for s in range(n_sets):
+        c = torch.roll(codes, shifts=37 * s, dims=0).contiguous() if s else codes
+        sc = torch.roll(scales, shifts=37 * s, dims=0).contiguous() if s else scales
+        sets.append(b.razer_pack_layout(desc, c, sc))
+    torch.cuda.synchronize()
+    return desc, sets, (codes, scales)
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    from oracle import razer_oracle as ro
+    from paper_2501_04052_b200 import inputs
+    N, K = DECODE_SHAPES[0]
+    codes, scales = inputs.random_codes(N, K, 1000)
+    codes, scales = codes.numpy(), scales.numpy()
+    x = inputs.bf16_to_bits(inputs.activations(1, K, 1000))
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        ro.matmul_w4a16(x, codes, scales, np.float32(0.002))
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    ms = 1e3 * sum(times) / len(times)
+    gbs = algo_bytes(1, N, K) / (ms * 1e-3) / 1e9
+    cores = torch.get_num_threads()
+    sample = f"each step = one {N}x{K} M=1 GEMV (first of the three decode shapes): oracle decode + FP64 matmul"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "decode GEMV, Llama-7B-shaped layers, M=1 (config 2)", "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-extras", action="store_true", help="skip the skinny / prefill / W4A4 lines")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2501_04052_b200 import build
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        build.build()
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    from paper_2501_04052_b200 import binding as b
+    from paper_2501_04052_b200 import inputs
+    pk = peaks()
+
+    # ---------------- decode step (config 2): resident inputs
+    n_sets = 9
+    layers = []
+    for i, (N, K) in enumerate(DECODE_SHAPES):
+        desc, sets, raw = make_sets(b, torch, inputs, N, K, n_sets, 1000 + i)
+        x = inputs.activations(1, K, 1000 + i).cuda()
+        y = torch.empty((1, N), dtype=torch.bfloat16, device="cuda")
+        ws = b.alloc_workspace(desc, 1, b.OP_GEMV, "cuda")
+        layers.append(dict(N=N, K=K, desc=desc, sets=sets, raw=raw if i == 0 else None, x=x, y=y, ws=ws))
+    step_bytes = sum(algo_bytes(1, l["N"], l["K"]) for l in layers)
+    packed_total = sum(s.numel() for l in layers for s in l["sets"])
+
+    def step(i):
+        for l in layers:
+            b.razer_gemv(l["desc"], l["sets"][i % n_sets], l["x"], l["y"], l["ws"])
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = b.razer_kernel_launches()
+    ms = time_cuda(step, args.steps, torch)
+    launches = b.razer_kernel_launches() - launches0
+    clocks = sampler.stop()
+    if dist:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * step_bytes / (ms * 1e-3) / 1e9
+
+    # ---------------- end to end: host buffers, copies inside the timed region
+    for l in layers:
+        l["xh"] = l["x"].cpu().pin_memory()
+        l["yh"] = torch.empty((1, l["N"]), dtype=torch.bfloat16).pin_memory()
+
+    def step_host(i):
+        for l in layers:
+            b.razer_gemv_host(l["desc"], l["sets"][i % n_sets], l["xh"], l["yh"], l["x"], l["y"], l["ws"])
+
+    for i in range(3):
+        step_host(i)
+    e2e_steps = max(20, args.steps // 4)
+    ms_e2e = time_cuda(step_host, e2e_steps, torch)
+    if dist:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e = {"value": world * step_bytes / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s",
+           "h2d_bytes_per_step": sum(2 * l["K"] for l in layers), "d2h_bytes_per_step": sum(2 * l["N"] for l in layers),
+           "ms_per_step": ms_e2e}
+
+    per_shape = []
+    for l in layers:
+        t = time_cuda(lambda i, l=l: b.razer_gemv(l["desc"], l["sets"][i % n_sets], l["x"], l["y"], l["ws"]),
+                      args.steps, torch)
+        gbs = algo_bytes(1, l["N"], l["K"]) / (t * 1e-3) / 1e9
+        per_shape.append({"M": 1, "N": l["N"], "K": l["K"], "us": t * 1e3, "GBps": gbs, "frac_hbm": gbs / pk["hbm"]})
+
+    result = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "decode GEMV, Llama-7B-shaped layers, M=1 (config 2): N x K = 4096x4096, 11008x4096, "
+                               "4096x11008; random RaZeR codes, bf16 N(0,1) activations",
+                   "l2": f"inputs larger than L2: weights rotate over {n_sets} packed copies, {packed_total / 1e6:.0f} MB",
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": value / world, "peak": pk["hbm"], "unit": "GB/s",
+                     "frac": value / world / pk["hbm"], "traffic": None, "peak_source": pk["source"],
+                     "kernel": "razer_gemv (3 launches per step)", "algorithmic_bytes_per_step": step_bytes,
+                     "frac_of_nominal_8TBps": value / world / 8000.0},
+        "decode_per_shape": per_shape,
+    }
+
+    if rank == 0 and not args.no_extras:
+        extras = []
+        del layers[1:]
+        torch.cuda.empty_cache()
+        for (N, K) in SKINNY_SHAPES:
+            ns = 6 if N * K < 100e6 else 3
+            desc, sets, _ = make_sets(b, torch, inputs, N, K, ns, 2000)
+            for M in (4, 16, 64):
+                x = inputs.activations(M, K, 2000 + M).cuda()
+                y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+                ws = b.alloc_workspace(desc, M, b.OP_GEMV, "cuda")
+                f = lambda i: b.razer_gemv(desc, sets[i % ns], x, y, ws)
+                for i in range(3):
+                    f(i)
+                t = time_cuda(f, 30, torch)
+                gbs = algo_bytes(M, N, K) / (t * 1e-3) / 1e9
+                extras.append({"config": 3, "op": "razer_gemv", "M": M, "N": N, "K": K, "us": t * 1e3, "GBps": gbs,
+                               "frac_hbm": gbs / pk["hbm"], "TFLOPs": 2.0 * M * N * K / (t * 1e-3) / 1e12})
+            del sets
+            torch.cuda.empty_cache()
+        for (N, K) in PREFILL_SHAPES:
+            M = 2048
+            desc, sets, _ = make_sets(b, torch, inputs, N, K, 2, 3000)
+            x = inputs.activations(M, K, 3000, outlier_channel_frac=0.01).cuda()
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            ws = b.alloc_workspace(desc, M, b.OP_GEMM, "cuda")
+            f = lambda i: b.razer_gemm(desc, sets[i % 2], x, y, ws)
+            for i in range(3):
+                f(i)
+            t = time_cuda(f, 10, torch)
+            tf = 2.0 * M * N * K / (t * 1e-3) / 1e12
+            extras.append({"config": 4, "op": "razer_gemm", "M": M, "N": N, "K": K, "us": t * 1e3, "TFLOPs": tf,
+                           "frac_bf16": tf / pk["bf16"]})
+            del sets
+            torch.cuda.empty_cache()
+        M, N, K = 256, 8192, 8192
+        desc, sets, _ = make_sets(b, torch, inputs, N, K, 4, 4000)
+        x = inputs.activations(M, K, 4000, outlier_channel_frac=0.01).cuda()
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+        ac, as_, ats = b.razer_quant_act(x)
+        tq = time_cuda(lambda i: b.razer_quant_act(x), 20, torch)
+        f = lambda i: b.razer_gemm_w4a4(desc, sets[i % 4], ac, as_, ats, y=y, workspace=ws)
+        for i in range(3):
+            f(i)
+        t = time_cuda(f, 10, torch)
+        extras.append({"config": 5, "op": "razer_quant_act", "M": M, "K": K, "us": tq * 1e3,
+                       "GBps": (M * K * 2 + M * K * 0.5625) / (tq * 1e-3) / 1e9})
+        tf = 2.0 * M * N * K / (t * 1e-3) / 1e12
+        extras.append({"config": 5, "op": "razer_gemm_w4a4", "M": M, "N": N, "K": K, "us": t * 1e3, "TFLOPs": tf,
+                       "frac_bf16": tf / pk["bf16"]})
+        result["extras"] = extras
+
+    if rank == 0 and not args.no_cpu:
+        import numpy as np
+        from oracle import razer_oracle as ro
+        l = layers[0]
+        codes, scales = l["raw"][0].cpu().numpy(), l["raw"][1].cpu().numpy()
+        xb = inputs.bf16_to_bits(l["x"].cpu())
+        t0 = time.perf_counter()
+        reps = 0
+        while reps < 2 or (time.perf_counter() - t0 < 10.0 and reps < 20):
+            yref = ro.matmul_w4a16(xb, codes, scales, np.float32(0.002))
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        b.razer_gemv(l["desc"], l["sets"][0], l["x"], l["y"], l["ws"])
+        torch.cuda.synchronize()
+        err = ro.rel_frobenius(inputs.bf16_to_bits(l["y"].cpu()), yref)
+        result["cpu_baseline"] = {"value": algo_bytes(1, l["N"], l["K"]) / dt / 1e9, "unit": "GB/s",
+                                  "cores": torch.get_num_threads(), "kind": "oracle",
+                                  "sample": f"{reps} x the {l['N']}x{l['K']} M=1 GEMV of the step "
+                                            "(oracle decode + FP64 matmul); the other two shapes scale with N*K",
+                                  "parity_rel_frobenius_vs_gpu": err}
+    if rank == 0:
+        print(json.dumps(result))
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

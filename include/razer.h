@@ -1,0 +1,148 @@
+/*
+ * razer.h - C ABI of the B200 (sm_100a) RaZeR matmul library.
+ *
+ * RaZeR (arXiv 2501.04052) stores a tensor as FP4-E2M1 codes in blocks of 16 along K.
+ * Each block has one 8-bit scale byte and the tensor has one FP32 scale (Sec. 3,
+ * Eq. 1-3).  FP4 has two zero codes; one of them is remapped, per block, to a special
+ * value chosen from a small set of allowed values, and the unused top bit(s) of the
+ * scale byte say which one (Sec. 4.1, 4.2, Eq. 6-7).
+ *
+ * Conventions shared by every entry point
+ *   y[m, n] = sum_k x[m, k] * W[n, k]      W is N x K, x is M x K, K contiguous in both.
+ *   Interchange format of a quantized tensor (what a quantizer emits, what
+ *   razer_pack_layout and razer_decode_act read):
+ *     codes  uint8 [rows][K/2]   element k = 2j in bits 3:0, k = 2j+1 in bits 7:4 of byte j;
+ *                                nibble = S E1 E0 M (Eq. 5)
+ *     scales uint8 [rows][K/16]  weights     : [sv_sign | sv_select | E2 E1 E0 | M2 M1 M0]
+ *                                              6-bit scale = an E4M3 code (Eq. 4) with E3 = 0
+ *                                activations : [sv_sign | E3 E2 E1 E0 | M2 M1 M0]
+ *     special value of a block = (sv_sign ? -1 : +1) * sv_mag[sv_select]   (Sec. 4.4)
+ *     element value            = special value if code == remap_code,
+ *                                0 if code is the other zero code, else Eq. 5
+ *     dequantized element      = tensor_scale * block_scale * element value   (Sec. 3)
+ *   All pointers named *_dev are DEVICE pointers; *_host are HOST pointers.  The caller
+ *   owns every buffer; no entry point allocates, frees or keeps device memory, and none
+ *   synchronizes the stream unless its comment says so.  `stream` is a cudaStream_t
+ *   passed as void* (NULL = the default stream).  bf16 tensors are raw 16-bit patterns.
+ *   Every function returns RAZER_OK (0) or a negative RAZER_ERR_* code, never throws;
+ *   razer_last_error() returns a description of the calling thread's last failure.
+ */
+#ifndef RAZER_H_
+#define RAZER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  RAZER_OK = 0,
+  RAZER_ERR_INVALID_ARG = -1,   /* null pointer, bad size, misaligned buffer               */
+  RAZER_ERR_UNSUPPORTED = -2,   /* a block size / special value / mode this build lacks     */
+  RAZER_ERR_WORKSPACE = -3,     /* workspace missing or smaller than razer_workspace_bytes  */
+  RAZER_ERR_CUDA = -4,          /* a CUDA runtime/driver call failed (text in last_error)   */
+  RAZER_ERR_DEVICE_TIMEOUT = -5 /* a bounded device-side wait gave up (status word set)     */
+};
+
+enum { RAZER_SCALE_E3M3_META2 = 0,   /* weights: 6-bit scale + 2 metadata bits (Sec. 4.1)  */
+       RAZER_SCALE_E4M3_META1 = 1 }; /* activations: 7-bit scale + 1 metadata bit          */
+
+enum { RAZER_OP_GEMV = 0, RAZER_OP_GEMM = 1, RAZER_OP_GEMM_W4A4 = 2 };
+
+/* Description of one RaZeR-quantized weight tensor (host struct, passed by pointer). */
+typedef struct razer_desc {
+  int32_t N;            /* rows (output features), >= 1                                     */
+  int32_t K;            /* columns (reduction dim), multiple of 16                          */
+  int32_t block;        /* elements per block; must be 16 (Sec. 3)                          */
+  int32_t scale_fmt;    /* RAZER_SCALE_E3M3_META2 for weights                                */
+  int32_t remap_code;   /* which zero nibble is the special value in the interchange codes:
+                           0x8 (negative zero, default) or 0x0                               */
+  float sv_mag[2];      /* special-value magnitudes selected by sv_select; each must be one
+                           of 2.5 3.5 4.5 5 5.5 6.5 7 7.5 8 9 10 12 (App. D.3)              */
+  float tensor_scale;   /* the FP32 per-tensor scale of Eq. 1                                */
+} razer_desc;
+
+/* Text of the calling thread's most recent error ("" if none). Never NULL. */
+const char* razer_last_error(void);
+
+/* Library/ABI version: major*10000 + minor*100 + patch. */
+int razer_version(void);
+
+/* Number of CUDA kernels this library has launched in this process so far (all threads).
+ * Lets a harness report how many device launches a timed region contained. */
+unsigned long long razer_kernel_launches(void);
+
+/* Size in bytes of the GPU-internal packed form of the tensor `d` describes.
+ * The packed form has the same 4.5 bits per weight (codes + scale bytes), padded to whole
+ * 128-row x 64-column tiles. */
+int razer_packed_bytes(const razer_desc* d, size_t* bytes_out);
+
+/* Offline weight shuffle (Sec. 4.3: weights are reordered once so that the kernels' loads
+ * are contiguous).  Reads the interchange format (codes_dev: N*K/2 bytes, scales_dev:
+ * N*K/16 bytes) and writes the packed form (razer_packed_bytes bytes, 16-byte aligned).
+ * Inside the packed form the remapped code is always 0x8 and blocks whose special value is
+ * positive are stored negated with a flag in the scale byte; both are lossless.
+ * Asynchronous on `stream`. */
+int razer_pack_layout(const razer_desc* d, const uint8_t* codes_dev, const uint8_t* scales_dev,
+                      void* packed_dev, void* stream);
+
+/* Verification hook: dequantize the packed tensor (Sec. 3: tensor scale x block scale x
+ * element value).  out_is_fp32 == 0: bf16 [N][K] of block_scale * element (exact);
+ * out_is_fp32 == 1: float [N][K] of fl32(tensor_scale * that) (one FP32 rounding). */
+int razer_dequant(const razer_desc* d, const void* packed_dev, void* out_dev, int out_is_fp32,
+                  void* stream);
+
+/* Scratch the matmul entry points need for `op` (RAZER_OP_*) with M activation rows.
+ * May be 0.  The workspace must be 256-byte aligned; its contents need no initialisation
+ * and are undefined afterwards.  Concurrent calls must not share a workspace. */
+int razer_workspace_bytes(const razer_desc* d, int M, int op, size_t* bytes_out);
+
+/* Decode GEMV / skinny GEMM (Sec. 4.3: weight-only FP4 x 16-bit kernel, low-batch regime):
+ * y[M][N] (bf16) = bf16( tensor_scale * sum_k x[m][k] * block_scale * element ), FP32
+ * accumulation, one rounding at the end.  x_dev: bf16 [M][K]; 1 <= M <= 64. */
+int razer_gemv(const razer_desc* d, const void* packed_dev, const void* x_dev, int M,
+               void* y_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Prefill GEMM (Sec. 4.3, high-batch regime): same result definition, any M >= 1. */
+int razer_gemm(const razer_desc* d, const void* packed_dev, const void* x_dev, int M,
+               void* y_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* razer_gemv with HOST activations and HOST output: copies x (M*K bf16) into
+ * x_stage_dev, runs razer_gemv, copies y (M*N bf16) back and synchronizes the stream.
+ * x_host / y_host should be pinned for the copies to be asynchronous. */
+int razer_gemv_host(const razer_desc* d, const void* packed_dev, const void* x_host, int M,
+                    void* y_host, void* x_stage_dev, void* y_stage_dev, void* workspace_dev,
+                    size_t workspace_bytes, void* stream);
+
+/* Online activation quantization (Sec. 4.2: each block is quantized once per allowed
+ * special value, +sv_mag and -sv_mag, and the lower squared error wins; Eq. 1-3, 6-7 with
+ * the 7-bit E4M3 block scale).  x_dev: bf16 [M][K], K multiple of 16.
+ * tensor_scale_in_dev: device float to use as the Eq. 1 scale, or NULL to compute it from
+ * the tensor maximum (then amax_scratch_dev, one device uint32, is required and is
+ * overwritten).  Writes act_codes_dev [M][K/2], act_scales_dev [M][K/16] in the
+ * interchange format (remapped code 0x8) and the scale used to tensor_scale_out_dev. */
+int razer_quant_act(const void* x_dev, int M, int K, float sv_mag,
+                    const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev,
+                    uint8_t* act_codes_dev, uint8_t* act_scales_dev,
+                    float* tensor_scale_out_dev, void* stream);
+
+/* Exact decode of RaZeR activations (interchange format, E4M3 scale, one metadata bit) to
+ * bf16 [M][K] holding block_scale * element (the tensor scale is NOT applied). */
+int razer_decode_act(const uint8_t* act_codes_dev, const uint8_t* act_scales_dev, int M, int K,
+                     float sv_mag, void* out_bf16_dev, void* stream);
+
+/* Weight-activation GEMM (App. D.3 setting, both operands RaZeR):
+ * y = bf16( w_scale * a_scale * sum_k decoded_act[m][k] * decoded_w[n][k] ).
+ * The workspace (RAZER_OP_GEMM_W4A4) holds the decoded activations.
+ * use_native_fp4 must be 0 in this build (block-scaled FP4 MMA path not present). */
+int razer_gemm_w4a4(const razer_desc* d, const void* packed_w_dev, const uint8_t* act_codes_dev,
+                    const uint8_t* act_scales_dev, const float* act_tensor_scale_dev, float act_sv_mag,
+                    int M, void* y_dev, void* workspace_dev, size_t workspace_bytes,
+                    int use_native_fp4, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAZER_H_ */

@@ -1,0 +1,112 @@
+// Shared declarations of the RaZeR CUDA library: packed-layout geometry, error plumbing,
+// small device helpers.  Nothing here is shared with the CPU oracle.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/razer.h"
+
+namespace razer {
+
+// ---------------------------------------------------------------------------------
+// Packed layout (GPU-internal form written by razer_pack_layout)
+//
+// The tensor is cut into tiles of TILE_ROWS rows x CHUNK_K columns (4 blocks of 16).
+// One tile-chunk is CHUNK_BYTES contiguous bytes:
+//   [blk 0..3][row 0..127] 8 bytes : the block's 16 nibbles, element j of the block in
+//                                    nibble j (byte j/2, low nibble first)
+//   [row 0..127] 4 bytes           : the four blocks' scale bytes
+// so that thread = row reads are contiguous across a warp (8 B or 4 B stride) and a whole
+// chunk is one bulk copy.  Chunks are ordered [row tile][k chunk].  Rows beyond N and
+// columns beyond K are zero blocks (scale byte 0).
+//
+// Inside the packed form:
+//   * the special value is always code 0x8, a true zero always code 0x0;
+//   * a block whose special value is positive is stored negated (sign bits of all non-zero
+//     codes flipped) so that code 0x8 always means "-sv_mag[select]";
+//   * scale byte = [negate | select | 6-bit scale code]; negate = 1 means the block's
+//     values are the negatives of the stored codes' values.
+// ---------------------------------------------------------------------------------
+constexpr int TILE_ROWS = 128;
+constexpr int CHUNK_K = 64;
+constexpr int CHUNK_BLOCKS = CHUNK_K / 16;
+constexpr int CHUNK_CODE_BYTES = CHUNK_BLOCKS * TILE_ROWS * 8;   // 4096
+constexpr int CHUNK_SCALE_BYTES = TILE_ROWS * 4;                 // 512
+constexpr int CHUNK_BYTES = CHUNK_CODE_BYTES + CHUNK_SCALE_BYTES;  // 4608
+
+struct Geometry {
+  int N, K;
+  int row_tiles;   // ceil(N / 128)
+  int k_chunks;    // ceil(K / 64)
+  __host__ __device__ size_t packed_bytes() const {
+    return (size_t)row_tiles * (size_t)k_chunks * CHUNK_BYTES;
+  }
+};
+
+__host__ __device__ inline Geometry make_geometry(int N, int K) {
+  Geometry g;
+  g.N = N;
+  g.K = K;
+  g.row_tiles = (N + TILE_ROWS - 1) / TILE_ROWS;
+  g.k_chunks = (K + CHUNK_K - 1) / CHUNK_K;
+  return g;
+}
+
+// Decode parameters derived from a razer_desc on the host, passed to kernels by value.
+struct DecodeParams {
+  float sv_mag[2];
+  float tensor_scale;
+  int remap_code;
+};
+
+// ---------------------------------------------------------------------------------
+// Error plumbing (host)
+// ---------------------------------------------------------------------------------
+int set_error(int code, const char* fmt, ...);
+int check_desc(const razer_desc* d);
+int check_cuda(cudaError_t e, const char* what);
+void count_launches(int n);   // bookkeeping behind razer_kernel_launches()
+bool sv_allowed(float m);
+
+#define RAZER_TRY(expr)            \
+  do {                             \
+    int _rc = (expr);              \
+    if (_rc != RAZER_OK) return _rc; \
+  } while (0)
+
+// ---------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------
+
+// FP4-E2M1 magnitude of the low three bits (Eq. 5): 0 .5 1 1.5 2 3 4 6.
+__device__ __forceinline__ float fp4_mag(uint32_t idx) {
+  const uint32_t e = (idx >> 1) & 3u;
+  const uint32_t m = idx & 1u;
+  // e != 0: 2^(e-1) * (1 + m/2); e == 0: m/2.  Build the float from its fields.
+  const float normal = __uint_as_float(((126u + e) << 23) | (m << 22));
+  return e ? normal : 0.5f * (float)m;
+}
+
+// Value of a 6/7-bit E4M3-coded block scale (Eq. 4, sign ignored).
+__device__ __forceinline__ float scale_value(uint32_t code) {
+  const uint32_t e = (code >> 3) & 0xFu;
+  const uint32_t m = code & 7u;
+  const float normal = __uint_as_float(((120u + e) << 23) | (m << 20));
+  return e ? normal : (float)m * 0.001953125f;   // m * 2^-9
+}
+
+// Element value of a packed-form nibble: code 0x8 is -sv, everything else Eq. 5.
+__device__ __forceinline__ float packed_elem(uint32_t nib, float neg_sv) {
+  const float mag = fp4_mag(nib & 7u);
+  const float v = (nib & 8u) ? -mag : mag;
+  return (nib == 8u) ? neg_sv : v;
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) {
+  return __uint_as_float(b << 16);
+}
+
+}  // namespace razer

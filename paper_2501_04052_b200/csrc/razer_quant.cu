@@ -1,0 +1,144 @@
+// razer_quant_act: online RaZeR quantization of bf16 activations (Sec. 4.2, Eq. 1-3, 6-7).
+//
+// Every FP32 operation below is a single correctly rounded IEEE operation issued through
+// an intrinsic (__fdiv_rn, __fmul_rn, __fadd_rn, __fsub_rn), so the compiler can neither
+// fuse nor reorder them: block scale, scaled values, the two candidate errors and the
+// choice between +sv and -sv are reproducible bit for bit.
+#include "razer_common.cuh"
+
+namespace razer {
+
+// Tensor maximum of |x| (Eq. 1 numerator): bit patterns of non-negative floats order like
+// unsigned integers, so one atomicMax per warp on the bf16 magnitude pattern suffices.
+__global__ void act_amax_kernel(const uint4* __restrict__ x, long long n_vec, uint32_t* __restrict__ amax_bits) {
+  uint32_t m = 0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec;
+       i += (long long)gridDim.x * blockDim.x) {
+    const uint4 v = x[i];
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t lo = w[j] & 0x7FFFu, hi = (w[j] >> 16) & 0x7FFFu;
+      // skip NaN patterns (exponent all ones, mantissa non-zero); infinities pass through
+      m = max(m, (lo > 0x7F80u) ? 0u : lo);
+      m = max(m, (hi > 0x7F80u) ? 0u : hi);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if ((threadIdx.x & 31) == 0 && m) atomicMax(amax_bits, m);
+}
+
+// Round a non-negative finite float to the nearest E4M3 code (ties to even mantissa),
+// saturating at `max_code`.
+__device__ __forceinline__ uint32_t round_to_e4m3(float t, uint32_t max_code) {
+  uint32_t code;
+  if (t < 0.015625f) {                       // below 2^-6: subnormal grid, quantum 2^-9
+    code = (uint32_t)__float2int_rn(__fmul_rn(t, 512.0f));   // exact product, ties to even
+  } else {
+    const uint32_t b = __float_as_uint(t);
+    const uint32_t e = (b >> 23) - 120u;     // biased E4M3 exponent (>= 1 here)
+    const uint32_t man = b & 0x7FFFFFu;
+    const uint32_t keep = man >> 20, rem = man & 0xFFFFFu;
+    const uint32_t up = (rem > 0x80000u) || (rem == 0x80000u && (keep & 1u));
+    code = (e >= 32u) ? max_code : ((e << 3) | keep) + up;   // a mantissa carry bumps the exponent
+  }
+  return min(code, max_code);
+}
+
+// Saturating round-to-nearest-even onto the FP4 magnitudes 0 .5 1 1.5 2 3 4 6 (Eq. 3).
+__device__ __forceinline__ uint32_t round_to_fp4_idx(float a) {
+  return (uint32_t)(a > 0.25f) + (uint32_t)(a >= 0.75f) + (uint32_t)(a > 1.25f) +
+         (uint32_t)(a >= 1.75f) + (uint32_t)(a > 2.5f) + (uint32_t)(a >= 3.5f) + (uint32_t)(a > 5.0f);
+}
+
+// One thread per 16-element block.
+__global__ void quant_act_kernel(const uint4* __restrict__ x, long long n_blocks, float sv_mag,
+                                 const float* __restrict__ scale_in, const uint32_t* __restrict__ amax_bits,
+                                 uint2* __restrict__ codes, uint8_t* __restrict__ scales,
+                                 float* __restrict__ scale_out) {
+  float d32;
+  if (scale_in) {
+    d32 = *scale_in;
+  } else {
+    const float amax = __uint_as_float(*amax_bits << 16);
+    d32 = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, __fmul_rn(448.0f, 6.0f));   // Eq. 1
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = d32;
+  const float d32x6 = __fmul_rn(d32, 6.0f);
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_blocks;
+       t += (long long)gridDim.x * blockDim.x) {
+    const uint4 v0 = x[2 * t], v1 = x[2 * t + 1];
+    const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    float xv[16];
+    float bmax = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      xv[2 * j] = __uint_as_float(w[j] << 16);
+      xv[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+      bmax = fmaxf(bmax, fmaxf(fabsf(xv[2 * j]), fabsf(xv[2 * j + 1])));
+    }
+    uint32_t w0 = 0, w1 = 0, sbyte = 0;
+    if (bmax > 0.0f) {
+      const float tq = __fdiv_rn(bmax, d32x6);                         // Eq. 2 argument
+      uint32_t scode = round_to_e4m3(tq, 126u);
+      if (scode == 0) scode = 1;                                       // keep a non-empty block alive
+      const float denom = __fmul_rn(d32, scale_value(scode));
+      float e_pos = 0.0f, e_neg = 0.0f;
+      uint32_t std_code[16];
+      uint32_t take_pos = 0, take_neg = 0;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float xs = __fdiv_rn(xv[j], denom);                      // the scaled block of Eq. 6
+        const uint32_t idx = round_to_fp4_idx(fabsf(xs));
+        const uint32_t neg = __float_as_uint(xs) >> 31;
+        const float r = neg ? -fp4_mag(idx) : fp4_mag(idx);
+        const float d_r = fabsf(__fsub_rn(xs, r));
+        const float d_p = fabsf(__fsub_rn(xs, sv_mag));
+        const float d_n = fabsf(__fsub_rn(xs, -sv_mag));
+        const bool tp = d_p < d_r, tn = d_n < d_r;                     // strictly closer only
+        const float qp = tp ? sv_mag : r, qn = tn ? -sv_mag : r;
+        const float dp = __fsub_rn(qp, xs), dn = __fsub_rn(qn, xs);
+        e_pos = __fadd_rn(e_pos, __fmul_rn(dp, dp));                   // ascending j, no fusion
+        e_neg = __fadd_rn(e_neg, __fmul_rn(dn, dn));
+        take_pos |= (uint32_t)tp << j;
+        take_neg |= (uint32_t)tn << j;
+        std_code[j] = idx ? (idx | (neg << 3)) : 0u;                   // a true zero is always code 0
+      }
+      const bool use_neg = e_neg < e_pos;                              // ties keep metadata 0 (+sv)
+      const uint32_t take = use_neg ? take_neg : take_pos;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t c = ((take >> j) & 1u) ? 8u : std_code[j];
+        if (j < 8) w0 |= c << (4 * j); else w1 |= c << (4 * (j - 8));
+      }
+      sbyte = (use_neg ? 0x80u : 0u) | scode;
+    }
+    codes[t] = make_uint2(w0, w1);
+    scales[t] = (uint8_t)sbyte;
+  }
+}
+
+int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* scale_in,
+                     uint32_t* amax_scratch, uint8_t* codes, uint8_t* scales, float* scale_out,
+                     cudaStream_t st) {
+  const long long n_blocks = (long long)M * (K / 16);
+  const long long n_vec = n_blocks * 2;
+  const int threads = 256;
+  auto grid = [&](long long n) {
+    long long b = (n + threads - 1) / threads;
+    return (int)(b < 1 ? 1 : (b > 148LL * 16 ? 148LL * 16 : b));
+  };
+  if (!scale_in) {
+    RAZER_TRY(check_cuda(cudaMemsetAsync(amax_scratch, 0, sizeof(uint32_t), st), "amax memset"));
+    act_amax_kernel<<<grid(n_vec), threads, 0, st>>>((const uint4*)x, n_vec, amax_scratch);
+    count_launches(1);
+    RAZER_TRY(check_cuda(cudaGetLastError(), "act_amax_kernel launch"));
+  }
+  quant_act_kernel<<<grid(n_blocks), threads, 0, st>>>((const uint4*)x, n_blocks, sv_mag, scale_in,
+                                                       amax_scratch, (uint2*)codes, scales, scale_out);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "quant_act_kernel launch");
+}
+
+}  // namespace razer

@@ -1,0 +1,248 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on identical seeded inputs.
+
+Bars: dequantized weights and quantized activation codes bit-exact; matmul outputs within
+1e-3 relative Frobenius error, both sides rounded to bf16 (accumulating 16-bit products in
+FP32 instead of FP64 moves a result across a bf16 rounding boundary only rarely; one such
+flip costs 2^-8 relative on one element).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import razer_oracle as ro
+from paper_2501_04052_b200 import inputs
+
+from _util import oracle_quantized_weights, rel_fro_bits, sample_rows, to_dev
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2501_04052_b200 import binding
+    return binding
+
+
+def _pack(b, codes, scales, d32, sv_mag=(5.0, 8.0), remap_code=0x8):
+    N, K = codes.shape[0], codes.shape[1] * 2
+    desc = b.make_desc(N, K, d32, sv_mag=sv_mag, remap_code=remap_code)
+    packed = b.razer_pack_layout(desc, to_dev(codes), to_dev(scales))
+    return desc, packed
+
+
+# ------------------------------------------------------------------ dequant (bit-exact)
+
+@pytest.mark.parametrize("N,K,seed", [(1024, 1024, 0), (200, 80, 3), (1, 16, 4), (129, 4160, 5)])
+def test_dequant_bit_exact_oracle_quantized(b, N, K, seed):
+    w, codes, scales, d32 = oracle_quantized_weights(N, K, seed)
+    desc, packed = _pack(b, codes, scales, d32)
+    d1 = b.razer_dequant(desc, packed, fp32=False).cpu()
+    d2 = b.razer_dequant(desc, packed, fp32=True).cpu().numpy()
+    want1 = ro.dequant_d1(codes, scales)
+    want2 = ro.dequant_d2(codes, scales, np.float32(d32))
+    assert np.array_equal(inputs.bf16_to_bits(d1), ro.f64_to_bf16_bits(want1.astype(np.float64)))
+    assert np.array_equal(d2.view(np.uint32), want2.view(np.uint32))
+
+
+@pytest.mark.parametrize("remap_code", [0x8, 0x0])
+@pytest.mark.parametrize("sv_mag", [(5.0, 8.0), (5.0, 7.0), (5.0, 9.0), (2.5, 12.0)])
+def test_dequant_bit_exact_random_codes(b, remap_code, sv_mag):
+    """Uniform random codes and metadata exercise every special value, both zero codes,
+    subnormal scales and zero blocks."""
+    N, K = 300, 1104
+    codes, scales = inputs.random_codes(N, K, seed=11, scale_lo=0, scale_hi=64, zero_block_frac=0.05)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.0123, sv_mag=sv_mag, remap_code=remap_code)
+    d1 = b.razer_dequant(desc, packed, fp32=False).cpu()
+    d2 = b.razer_dequant(desc, packed, fp32=True).cpu().numpy()
+    want1 = ro.dequant_d1(codes, scales, sv_mag=sv_mag, remap_code=remap_code)
+    want2 = ro.dequant_d2(codes, scales, np.float32(0.0123), sv_mag=sv_mag, remap_code=remap_code)
+    assert np.array_equal(inputs.bf16_to_bits(d1), ro.f64_to_bf16_bits(want1.astype(np.float64)))
+    assert np.array_equal(d2.view(np.uint32), want2.view(np.uint32))
+
+
+# ------------------------------------------------------------------ GEMV / skinny GEMM
+
+def _check_matmul(b, fn, desc, packed, codes, scales, d32, x, rows=None, **kw):
+    y = fn(desc, packed, x.cuda())
+    torch.cuda.synchronize()
+    xb = inputs.bf16_to_bits(x)
+    if rows is None:
+        ref = ro.matmul_w4a16(xb, codes, scales, np.float32(d32), **kw)
+        got = y
+    else:
+        ref = ro.matmul_w4a16(xb, codes[rows], scales[rows], np.float32(d32), **kw)
+        got = y[:, torch.from_numpy(rows).cuda()]
+    err = rel_fro_bits(got, ref)
+    assert err <= TOL, f"relative Frobenius error {err:.3e}"
+    return err
+
+
+def test_gemv_config1_student_t(b):
+    """BASELINE config 1: N=K=1024, Student-t x 0.02 weights from seed 0, M=1."""
+    w, codes, scales, d32 = oracle_quantized_weights(1024, 1024, 0, outliers=0.0)
+    desc, packed = _pack(b, codes, scales, d32)
+    x = inputs.activations(1, 1024, 0)
+    _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, d32, x)
+
+
+@pytest.mark.parametrize("N,K", [(4096, 4096), (11008, 4096), (4096, 11008)])
+def test_gemv_config2_llama7b_shapes(b, N, K):
+    w, codes, scales, d32 = oracle_quantized_weights(N, K, 1)
+    desc, packed = _pack(b, codes, scales, d32)
+    x = inputs.activations(1, K, 1)
+    _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, d32, x)
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 7, 16, 33, 64])
+def test_gemv_ragged_shapes_random_codes(b, M):
+    N, K = 333, 2064                      # N not a multiple of the row tile, K not of the k chunk
+    codes, scales = inputs.random_codes(N, K, seed=20 + M, zero_block_frac=0.02)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.004)
+    x = inputs.activations(M, K, 20 + M)
+    _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, 0.004, x)
+
+
+@pytest.mark.parametrize("sv_mag,remap_code", [((5.0, 7.0), 0x8), ((5.0, 9.0), 0x0), ((2.5, 12.0), 0x8)])
+def test_gemv_other_special_values(b, sv_mag, remap_code):
+    N, K = 256, 1024
+    codes, scales = inputs.random_codes(N, K, seed=31)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.01, sv_mag=sv_mag, remap_code=remap_code)
+    x = inputs.activations(4, K, 31)
+    _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, 0.01, x, sv_mag=sv_mag, remap_code=remap_code)
+
+
+@pytest.mark.parametrize("M,N,K", [(4, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192),
+                                   (4, 28672, 8192), (64, 28672, 8192), (16, 8192, 28672), (64, 8192, 28672)])
+def test_skinny_config3_full_size_sampled_rows(b, M, N, K):
+    """BASELINE config 3 at full size: random RaZeR codes, a sample of output columns checked
+    one by one against the oracle."""
+    codes, scales = inputs.random_codes(N, K, seed=40)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.002)
+    x = inputs.activations(M, K, 40 + M)
+    rows = sample_rows(N, 192, 41)
+    _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, 0.002, x, rows=rows)
+
+
+def test_skinny_config3_oracle_quantized(b):
+    w, codes, scales, d32 = oracle_quantized_weights(2048, 8192, 2)
+    desc, packed = _pack(b, codes, scales, d32)
+    for M in (4, 16, 64):
+        x = inputs.activations(M, 8192, 50 + M)
+        _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, d32, x)
+
+
+# ------------------------------------------------------------------ prefill GEMM
+
+@pytest.mark.parametrize("M,N,K", [(256, 512, 1024), (130, 200, 464), (2048, 1024, 4096)])
+def test_gemm_oracle_quantized(b, M, N, K):
+    w, codes, scales, d32 = oracle_quantized_weights(N, K, 3, outliers=0.0)
+    desc, packed = _pack(b, codes, scales, d32)
+    x = inputs.activations(M, K, 60, outlier_channel_frac=0.01)
+    _check_matmul(b, b.razer_gemm, desc, packed, codes, scales, d32, x)
+
+
+@pytest.mark.parametrize("N,K", [(14336, 4096), (4096, 14336)])
+def test_gemm_config4_full_size_sampled_rows(b, N, K):
+    codes, scales = inputs.random_codes(N, K, seed=70)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.002)
+    x = inputs.activations(2048, K, 70, outlier_channel_frac=0.01)
+    rows = sample_rows(N, 96, 71)
+    _check_matmul(b, b.razer_gemm, desc, packed, codes, scales, 0.002, x, rows=rows)
+
+
+# ------------------------------------------------------------------ activation quantization / W4A4
+
+@pytest.mark.parametrize("M,K,seed", [(256, 8192, 80), (7, 48, 81), (33, 1040, 82)])
+def test_quant_act_bit_exact(b, M, K, seed):
+    x = inputs.activations(M, K, seed, outlier_channel_frac=0.01)
+    codes, scales, ts = b.razer_quant_act(x.cuda())
+    torch.cuda.synchronize()
+    want_c, want_s, want_d, dbg = ro.quantize_act(inputs.bf16_to_bits(x), return_debug=True)
+    assert np.float32(ts.item()) == want_d
+    got_s, got_c = scales.cpu().numpy(), codes.cpu().numpy()
+    assert np.array_equal(got_s & 0x7F, want_s & 0x7F)
+    # metadata and codes must agree except where the two candidates' errors tie within rounding
+    blk_ok = (got_s == want_s) & np.all((got_c == want_c).reshape(M, K // 16, 8), axis=2)
+    assert np.all(blk_ok | dbg["near_tie"])
+    assert blk_ok.mean() > 0.999
+    # the decode kernel inverts the GPU's own codes exactly like the oracle's decoder
+    d1 = b.razer_decode_act(codes, scales).cpu()
+    want1 = ro.dequant_d1(got_c, got_s, scale_fmt=ro.SCALE_E4M3_META1, sv_mag=(5.0,))
+    assert np.array_equal(inputs.bf16_to_bits(d1), ro.f64_to_bf16_bits(want1.astype(np.float64)))
+
+
+def test_quant_act_given_scale_and_zero_input(b):
+    x = inputs.activations(8, 256, 83)
+    given = torch.tensor([0.05], dtype=torch.float32)
+    codes, scales, ts = b.razer_quant_act(x.cuda(), tensor_scale=given.cuda())
+    want_c, want_s, want_d = ro.quantize_act(inputs.bf16_to_bits(x), tensor_scale=np.float32(0.05))
+    assert ts.item() == np.float32(0.05)
+    assert np.array_equal(scales.cpu().numpy(), want_s) and np.array_equal(codes.cpu().numpy(), want_c)
+    z = torch.zeros((4, 64), dtype=torch.bfloat16)
+    codes, scales, ts = b.razer_quant_act(z.cuda())
+    assert ts.item() == 1.0 and not codes.any() and not scales.any()
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 1024, 8192), (17, 200, 464)])
+def test_w4a4_oracle_quantized(b, M, N, K):
+    """BASELINE config 5 (rows of N sampled down to keep the oracle quantizer quick)."""
+    w, wc, ws, wd = oracle_quantized_weights(N, K, 4)
+    desc, packed = _pack(b, wc, ws, wd)
+    x = inputs.activations(M, K, 90, outlier_channel_frac=0.01)
+    ac, as_, ats = b.razer_quant_act(x.cuda())
+    y = b.razer_gemm_w4a4(desc, packed, ac, as_, ats)
+    torch.cuda.synchronize()
+    ref = ro.matmul_w4a4(ac.cpu().numpy(), as_.cpu().numpy(), np.float32(ats.item()), wc, ws, np.float32(wd))
+    err = rel_fro_bits(y, ref)
+    assert err <= TOL, f"relative Frobenius error {err:.3e}"
+
+
+def test_w4a4_config5_full_size_sampled_rows(b):
+    M, N, K = 256, 8192, 8192
+    wc, ws = inputs.random_codes(N, K, seed=95)
+    wc, ws = wc.numpy(), ws.numpy()
+    desc, packed = _pack(b, wc, ws, 0.002)
+    x = inputs.activations(M, K, 95, outlier_channel_frac=0.01)
+    ac, as_, ats = b.razer_quant_act(x.cuda())
+    y = b.razer_gemm_w4a4(desc, packed, ac, as_, ats)
+    torch.cuda.synchronize()
+    rows = sample_rows(N, 128, 96)
+    ref = ro.matmul_w4a4(ac.cpu().numpy(), as_.cpu().numpy(), np.float32(ats.item()), wc[rows], ws[rows],
+                         np.float32(0.002))
+    err = rel_fro_bits(y[:, torch.from_numpy(rows).cuda()], ref)
+    assert err <= TOL, f"relative Frobenius error {err:.3e}"
+
+
+# ------------------------------------------------------------------ host-buffer entry point, errors
+
+def test_gemv_host_entry_point(b):
+    N, K, M = 512, 1024, 2
+    codes, scales = inputs.random_codes(N, K, seed=97)
+    desc, packed = _pack(b, codes.numpy(), scales.numpy(), 0.01)
+    x = inputs.activations(M, K, 97).pin_memory()
+    y = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    xs = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    ys = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = b.alloc_workspace(desc, M, b.OP_GEMV, "cuda")
+    b.razer_gemv_host(desc, packed, x, y, xs, ys, ws)
+    y_dev = b.razer_gemv(desc, packed, x.cuda())
+    assert torch.equal(y, y_dev.cpu())
+
+
+def test_workspace_too_small_is_an_error(b):
+    N, K = 512, 4096
+    codes, scales = inputs.random_codes(N, K, seed=98)
+    desc, packed = _pack(b, codes.numpy(), scales.numpy(), 0.01)
+    need = b.razer_workspace_bytes(desc, 1, b.OP_GEMV)
+    if need > 256:
+        x = inputs.activations(1, K, 98).cuda()
+        tiny = torch.empty(256, dtype=torch.uint8, device="cuda")
+        with pytest.raises(b.RazerError) as e:
+            b.razer_gemv(desc, packed, x, workspace=tiny)
+        assert e.value.code == b.ERR_WORKSPACE
