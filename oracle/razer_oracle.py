@@ -347,10 +347,11 @@ def decode_block_values(codes, scales, scale_fmt=SCALE_E3M3_META2, sv_mag=(5.0, 
 
 
 def dequant_d1(codes, scales, **kw):
-    """D1 = q * Delta8 (exact; fits bf16).  Returned as float32."""
+    """D1 = q * Delta8 (exact; fits bf16).  Returned as float32.  A zero product is
+    written as +0 (the sign of a zero carries no information in the format)."""
     block = kw.get("block", BLOCK)
     q, s = decode_block_values(codes, scales, **kw)
-    return (q * np.repeat(s, block, axis=1)).astype(np.float32)
+    return (q * np.repeat(s, block, axis=1) + 0.0).astype(np.float32)
 
 
 def dequant_d2(codes, scales, tensor_scale, **kw):
