@@ -95,9 +95,22 @@ int razer_dequant(const razer_desc* d, const void* packed_dev, void* out_dev, in
                   void* stream);
 
 /* Scratch the matmul entry points need for `op` (RAZER_OP_*) with M activation rows.
- * May be 0.  The workspace must be 256-byte aligned; its contents need no initialisation
- * and are undefined afterwards.  Concurrent calls must not share a workspace. */
+ * The workspace must be 256-byte aligned and must have been prepared once with
+ * razer_workspace_init; the matmul calls leave it prepared, so one workspace can serve any
+ * number of calls, shapes included, one after another.  Calls that may overlap on the GPU
+ * must not share a workspace. */
 int razer_workspace_bytes(const razer_desc* d, int M, int op, size_t* bytes_out);
+
+/* Prepare a workspace: clears the status word and the per-tile arrival counters the
+ * stripe reduction (Sec. 4.3, App. E: partial results of stripes are combined through
+ * global memory) relies on.  Needed once after allocation, and again after a call returned
+ * RAZER_ERR_DEVICE_TIMEOUT or the process was interrupted mid-kernel.  Asynchronous. */
+int razer_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Synchronizes `stream` and reads the workspace's device status word: RAZER_OK, or
+ * RAZER_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded wait (its output is then
+ * undefined; razer_last_error names the wait). */
+int razer_workspace_status(const void* workspace_dev, void* stream);
 
 /* Decode GEMV / skinny GEMM (Sec. 4.3: weight-only FP4 x 16-bit kernel, low-batch regime):
  * y[M][N] (bf16) = bf16( tensor_scale * sum_k x[m][k] * block_scale * element ), FP32

@@ -23,7 +23,7 @@ OP_GEMV, OP_GEMM, OP_GEMM_W4A4 = 0, 1, 2
 
 EXPORTS = (
     "razer_last_error", "razer_version", "razer_kernel_launches", "razer_packed_bytes", "razer_pack_layout", "razer_dequant",
-    "razer_workspace_bytes", "razer_gemv", "razer_gemm", "razer_gemv_host", "razer_quant_act",
+    "razer_workspace_bytes", "razer_workspace_init", "razer_workspace_status", "razer_gemv", "razer_gemm", "razer_gemv_host", "razer_quant_act",
     "razer_decode_act", "razer_gemm_w4a4",
 )
 
@@ -52,6 +52,8 @@ _lib.razer_packed_bytes.argtypes = [POINTER(RazerDesc), POINTER(c_size_t)]
 _lib.razer_pack_layout.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_void_p, c_void_p]
 _lib.razer_dequant.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_void_p]
 _lib.razer_workspace_bytes.argtypes = [POINTER(RazerDesc), c_int, c_int, POINTER(c_size_t)]
+_lib.razer_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
+_lib.razer_workspace_status.argtypes = [c_void_p, c_void_p]
 _lib.razer_gemv.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
 _lib.razer_gemm.argtypes = _lib.razer_gemv.argtypes
 _lib.razer_gemv_host.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
@@ -134,9 +136,21 @@ def razer_dequant(desc: RazerDesc, packed: torch.Tensor, fp32: bool) -> torch.Te
     return out
 
 
-def alloc_workspace(desc: RazerDesc, M: int, op: int, device) -> torch.Tensor | None:
+def razer_workspace_init(workspace: torch.Tensor) -> None:
+    _check(_lib.razer_workspace_init(_ptr(workspace), workspace.numel(), _stream()))
+
+
+def razer_workspace_status(workspace: torch.Tensor) -> None:
+    """Synchronizes the stream; raises RazerError(ERR_DEVICE_TIMEOUT) if a kernel gave up a wait."""
+    _check(_lib.razer_workspace_status(_ptr(workspace), _stream()))
+
+
+def alloc_workspace(desc: RazerDesc, M: int, op: int, device) -> torch.Tensor:
+    """Allocate (torch) and prepare (razer_workspace_init) a workspace for `op` with M rows."""
     n = razer_workspace_bytes(desc, M, op)
-    return torch.empty(max(n, 256), dtype=torch.uint8, device=device)
+    ws = torch.empty(max(n, 256), dtype=torch.uint8, device=device)
+    razer_workspace_init(ws)
+    return ws
 
 
 def _matmul(fn, desc, packed, x, y, workspace, op):

@@ -136,6 +136,22 @@ int razer_workspace_bytes(const razer_desc* d, int M, int op, size_t* bytes_out)
   return RAZER_OK;
 }
 
+int razer_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream) {
+  RAZER_TRY(check_ptr(workspace_dev, 256, "workspace_dev"));
+  if (workspace_bytes == 0) return RAZER_OK;
+  return check_cuda(cudaMemsetAsync(workspace_dev, 0, workspace_bytes, (cudaStream_t)stream), "workspace memset");
+}
+
+int razer_workspace_status(const void* workspace_dev, void* stream) {
+  RAZER_TRY(check_ptr(workspace_dev, 256, "workspace_dev"));
+  uint32_t st = 0;
+  RAZER_TRY(check_cuda(cudaMemcpyAsync(&st, workspace_dev, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream),
+                       "status copy"));
+  RAZER_TRY(check_cuda(cudaStreamSynchronize((cudaStream_t)stream), "stream synchronize"));
+  if (st != 0) return set_error(RAZER_ERR_DEVICE_TIMEOUT, "a device-side wait gave up (wait id %u)", st);
+  return RAZER_OK;
+}
+
 static int matmul_common(const razer_desc* d, const void* packed_dev, const void* x_dev, int M, void* y_dev,
                          void* ws, size_t ws_bytes, float extra_scale, const float* extra_scale_dev,
                          cudaStream_t st) {
@@ -182,6 +198,7 @@ int razer_gemv_host(const razer_desc* d, const void* packed_dev, const void* x_h
                           nullptr, st));
   RAZER_TRY(check_cuda(cudaMemcpyAsync(y_host, y_stage_dev, (size_t)M * d->N * 2, cudaMemcpyDeviceToHost, st),
                        "copy of y to the host"));
+  if (workspace_dev) return razer_workspace_status(workspace_dev, stream);   // synchronizes
   return check_cuda(cudaStreamSynchronize(st), "stream synchronize");
 }
 

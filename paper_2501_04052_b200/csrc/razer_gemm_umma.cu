@@ -1,14 +1,569 @@
-// Tensor-core (tcgen05 / TMEM) matmul against packed RaZeR weights.  Placeholder until the
-// kernel lands: reports every shape as unsupported so the CUDA-core kernel is used.
+// Tensor-core matmul against packed RaZeR weights for sm_100a (tcgen05 + TMEM + TMA).
+//
+//   y[m, n] = bf16( ts * sum_k x[m, k] * D1[n, k] ),   D1 = block_scale * element (exact bf16)
+//
+// Mapping onto the 5th-generation tensor core: the weight tile is the MMA's A operand
+// (128 weight rows = 128 TMEM lanes), the activation tile is the B operand (NT tokens,
+// K-major in shared memory, 128-byte swizzle, written by TMA), the accumulator D[128 x NT]
+// lives in TMEM.  Weights never exist as bf16 in shared or global memory: a TMA bulk copy
+// brings the packed 4.5-bit chunk into shared memory, four "dequant" warps (thread = weight
+// row) decode one 16-element block at a time in registers and write the bf16 pairs straight
+// into TMEM with tcgen05.st, and the MMA reads A from TMEM.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..5 = dequant, then epilogue of the tile they just fed.
+//
+// Work partition (Sec. 4.3 / App. E of the paper: stripes of about equal length that may span
+// several output tiles, partial results reduced through global memory): the grid is
+// persistent, work items are (output tile, k-stage) pairs in tile-major order and every CTA
+// takes one contiguous stripe of items.  A stripe's first and last tile may be partial; those
+// go to a per-CTA FP32 slot in the workspace and the last CTA to arrive at a tile (one
+// counter per tile) adds the slots in CTA order, scales and rounds once.  Tiles a stripe
+// covers completely are written directly.
+//
+// Every wait (mbarrier, counter) is bounded: on expiry the thread records a code in the
+// workspace status word and the kernel drains and exits instead of hanging the GPU.
+#include <cuda.h>
+#include <cstdlib>
+
 #include "razer_common.cuh"
 
 namespace razer {
 
-bool umma_supported(const razer_desc*, int) { return false; }
-size_t umma_workspace_bytes(const razer_desc*, int) { return 0; }
-int launch_gemm_umma(const razer_desc*, const void*, const void*, int, int, float, const float*, void*, void*,
-                     size_t, cudaStream_t) {
-  return set_error(RAZER_ERR_UNSUPPORTED, "tensor-core kernel not built");
+// ------------------------------------------------------------------ workspace layout
+constexpr size_t WS_STATUS_BYTES = 256;               // word 0: device status (0 = ok)
+constexpr int UMMA_THREADS = 192;
+constexpr uint32_t WAIT_LIMIT = 1u << 26;             // try_wait rounds before giving up, and
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;     // wall-clock bound of one wait (2 s)
+
+static size_t align256(size_t v) { return (v + 255) / 256 * 256; }
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false = gave up (or another thread already flagged a failure).
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t i = 1; i < WAIT_LIMIT; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+    }
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(v[0]),
+               "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored with the 128-byte swizzle:
+// rows are 128 bytes (64 elements), groups of 8 rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_b_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024u >> 4) << 32;                 // stride byte offset: 8 rows x 128 B
+  d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                            // swizzle mode: 128 B
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> f32, both operands K-major, M = 128, N = NT.
+__host__ __device__ constexpr uint32_t make_idesc(int nt) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ decode (registers)
+// One packed block (16 nibbles + scale byte) -> 8 registers of two bf16 each, element 2p in
+// the low half of register p.  block_scale * element has at most 8 significant bits, so the
+// FP32 product's upper 16 bits are the exact bf16.
+__device__ __forceinline__ void decode_block_bf16(uint2 cw, uint32_t sb, float neg_sv0, float neg_sv1,
+                                                  uint32_t (&out)[8]) {
+  float s = scale_value(sb & 0x3Fu);
+  if (sb & 0x80u) s = -s;
+  const float neg_sv = (sb & 0x40u) ? neg_sv1 : neg_sv0;
+#pragma unroll
+  for (int p = 0; p < 8; ++p) {
+    const uint32_t w = (p < 4) ? cw.x : cw.y;
+    const uint32_t byte = (w >> (8 * (p & 3))) & 0xFFu;
+    const float a = packed_elem(byte & 0xFu, neg_sv) * s;
+    const float b = packed_elem(byte >> 4, neg_sv) * s;
+    out[p] = (__float_as_uint(a) >> 16) | (__float_as_uint(b) & 0xFFFF0000u);
+  }
+}
+
+// ------------------------------------------------------------------ kernel
+struct UmmaArgs {
+  const uint8_t* packed;
+  __nv_bfloat16* y;
+  float* slots;              // [grid][2][NT][128] FP32 partial tiles
+  uint32_t* counters;        // one per output tile, zero between calls
+  uint32_t* status;          // device status word
+  const float* extra_scale;  // optional device scalar multiplied into the tensor scale
+  Geometry g;
+  float neg_sv0, neg_sv1, tensor_scale;
+  int M, token_tiles, steps_per_tile;
+  long long total_items;
+};
+
+template <int NT, int CH, int STAGES, int ASTAGES>
+struct UmmaCfg {
+  static constexpr int W_BYTES = CH * CHUNK_BYTES;
+  static constexpr int X_BOX_BYTES = NT * 128;                 // NT tokens x 64 k x 2 B
+  static constexpr int X_BYTES = CH * X_BOX_BYTES;
+  static constexpr int W_PAD = (W_BYTES + 1023) / 1024 * 1024; // keep the x boxes 1024-byte aligned
+  static constexpr int STAGE_BYTES = W_PAD + X_BYTES;
+  static constexpr int ACC_COLS = NT < 32 ? 32 : NT;
+  static constexpr int A_STAGE_COLS = CH * 32;                 // 4 blocks x 8 columns per chunk
+  static constexpr int TMEM_COLS_NEEDED = ACC_COLS + ASTAGES * A_STAGE_COLS;
+  static constexpr int TMEM_COLS = TMEM_COLS_NEEDED <= 64 ? 64 : TMEM_COLS_NEEDED <= 128 ? 128
+                                   : TMEM_COLS_NEEDED <= 256 ? 256 : 512;
+  static constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 3;
+  static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + NUM_BARS * 8 + 64;
+  static_assert(TMEM_COLS_NEEDED <= 512, "TMEM budget exceeded");
+  static_assert(NT % 16 == 0 && NT >= 16 && NT <= 256, "UMMA N for M = 128");
+};
+
+__device__ __forceinline__ int cta_of_item(long long item, int grid, long long total) {
+  return (int)((((item + 1) * grid) - 1) / total);
+}
+
+template <int NT, int CH, int STAGES, int ASTAGES>
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) {
+  using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * Cfg::STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + Cfg::NUM_BARS);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  uint32_t* bcast = tmem_slot + 2;                      // epilogue broadcast word
+
+  const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> dequant, MMA
+  const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]  MMA commit -> TMA
+  const uint32_t bar_afull = bar_empty + 8 * STAGES;    // [ASTAGES] dequant -> MMA
+  const uint32_t bar_aempty = bar_afull + 8 * ASTAGES;  // [ASTAGES] MMA commit -> dequant
+  const uint32_t bar_accfull = bar_aempty + 8 * ASTAGES;
+  const uint32_t bar_accempty = bar_accfull + 8;
+  const uint32_t bar_epi = bar_accempty + 8;            // rendezvous of the 128 epilogue threads
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grid = gridDim.x, cta = blockIdx.x;
+  const long long it_begin = (a.total_items * cta) / grid;
+  const long long it_end = (a.total_items * (cta + 1)) / grid;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < ASTAGES; ++i) {
+      mbar_init(bar_afull + 8 * i, 128);
+      mbar_init(bar_aempty + 8 * i, 1);
+    }
+    mbar_init(bar_accfull, 1);
+    mbar_init(bar_accempty, 128);
+    mbar_init(bar_epi, 128);
+    *abort_flag = 0;
+    tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_a0 = tmem_base + Cfg::ACC_COLS;
+
+  auto fail = [&](uint32_t code) {
+    *abort_flag = 1;
+    atomicCAS(a.status, 0u, code);
+  };
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+      long long issued = 0;
+      for (long long it = it_begin; it < it_end; ++it, ++issued) {
+        const int s = (int)(issued % STAGES);
+        const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
+        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { fail(1); break; }
+        const long long tile = it / a.steps_per_tile;
+        const int step = (int)(it % a.steps_per_tile);
+        const int rt = (int)(tile / a.token_tiles), tt = (int)(tile % a.token_tiles);
+        const int c0 = step * CH;
+        const int nch = min(CH, a.g.k_chunks - c0);
+        uint8_t* st = smem + (size_t)s * Cfg::STAGE_BYTES;
+        mbar_expect_tx(bar_full + 8 * s, (uint32_t)(nch * (CHUNK_BYTES + Cfg::X_BOX_BYTES)));
+        bulk_copy_g2s(smem_u32(st), a.packed + ((size_t)rt * a.g.k_chunks + c0) * CHUNK_BYTES,
+                      (uint32_t)(nch * CHUNK_BYTES), bar_full + 8 * s);
+        for (int c = 0; c < nch; ++c)
+          tma_load_2d(smem_u32(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES), &tmap_x, (c0 + c) * CHUNK_K, tt * NT,
+                      bar_full + 8 * s);
+      }
+      // Drain: copies still in flight must land before this CTA's shared memory is released.
+      const long long pending = issued < STAGES ? issued : STAGES;
+      for (long long f = issued - pending; f < issued; ++f)
+        mbar_wait(bar_full + 8 * (int)(f % STAGES), (uint32_t)((f / STAGES) & 1), tmem_slot + 3);
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(NT);
+      long long n = 0, seg = 0;
+      for (long long it = it_begin; it < it_end; ++it, ++n) {
+        const int s = (int)(n % STAGES), t = (int)(n % ASTAGES);
+        const uint32_t ph = (uint32_t)((n / STAGES) & 1), aph = (uint32_t)((n / ASTAGES) & 1);
+        const long long tile = it / a.steps_per_tile;
+        const int step = (int)(it % a.steps_per_tile);
+        const bool seg_first = (it == it_begin) || step == 0;
+        const bool seg_last = (it + 1 == it_end) || step == a.steps_per_tile - 1;
+        const int nch = min(CH, a.g.k_chunks - step * CH);
+        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { fail(2); break; }
+        if (!mbar_wait(bar_afull + 8 * t, aph, abort_flag)) { fail(3); break; }
+        if (seg_first && !mbar_wait(bar_accempty, (uint32_t)((seg & 1) ^ 1), abort_flag)) { fail(4); break; }
+        tc_fence_after();
+        const uint32_t xs = smem_u32(smem + (size_t)s * Cfg::STAGE_BYTES + Cfg::W_PAD);
+        const uint32_t a_t = tmem_a0 + t * Cfg::A_STAGE_COLS;
+        for (int j = 0; j < nch * 4; ++j) {
+          const uint64_t bd = make_b_desc(xs + (j >> 2) * Cfg::X_BOX_BYTES + (j & 3) * 32);
+          tc_mma_ts(tmem_base, a_t + j * 8, bd, idesc, (seg_first && j == 0) ? 0u : 1u);
+        }
+        tc_commit(bar_empty + 8 * s);
+        tc_commit(bar_aempty + 8 * t);
+        if (seg_last) {
+          tc_commit(bar_accfull);
+          ++seg;
+        }
+        (void)tile;
+      }
+    }
+  } else {
+    // ===================== dequant + epilogue (128 threads, thread = weight row) =====================
+    const int row = 32 * (warp & 3) + lane;              // TMEM lane this thread owns
+    const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
+    const bool leader = (threadIdx.x == 64);
+    const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
+    long long n = 0, seg = 0;
+    uint32_t epi_phase = 0;
+    // all 32 lanes take the same branch after a wait, so the .aligned tcgen05 instructions stay convergent
+    auto wait_all = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
+      const bool got = mbar_wait(bar, parity, abort_flag);
+      if (!got) fail(code);
+      return __all_sync(0xFFFFFFFFu, got);
+    };
+    auto epi_sync = [&]() -> bool {                     // bounded rendezvous of the epilogue threads
+      mbar_arrive(bar_epi);
+      const bool got = wait_all(bar_epi, epi_phase & 1u, 8);
+      ++epi_phase;
+      return got;
+    };
+    for (long long it = it_begin; it < it_end; ++it, ++n) {
+      const int s = (int)(n % STAGES), t = (int)(n % ASTAGES);
+      const uint32_t ph = (uint32_t)((n / STAGES) & 1), aph = (uint32_t)((n / ASTAGES) & 1);
+      const long long tile = it / a.steps_per_tile;
+      const int step = (int)(it % a.steps_per_tile);
+      const bool seg_last = (it + 1 == it_end) || step == a.steps_per_tile - 1;
+      const int nch = min(CH, a.g.k_chunks - step * CH);
+      if (!wait_all(bar_full + 8 * s, ph, 5)) break;
+      if (!wait_all(bar_aempty + 8 * t, aph ^ 1u, 6)) break;
+      tc_fence_after();
+      const uint8_t* st = smem + (size_t)s * Cfg::STAGE_BYTES;
+      const uint32_t a_t = tmem_a0 + t * Cfg::A_STAGE_COLS + lane_off;
+      for (int c = 0; c < nch; ++c) {
+        const uint8_t* ck = st + c * CHUNK_BYTES;
+        const uint32_t sw = *reinterpret_cast<const uint32_t*>(ck + CHUNK_CODE_BYTES + row * 4);
+#pragma unroll
+        for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
+          const uint2 cw = *reinterpret_cast<const uint2*>(ck + (blk * TILE_ROWS + row) * 8);
+          uint32_t v[8];
+          decode_block_bf16(cw, (sw >> (8 * blk)) & 0xFFu, a.neg_sv0, a.neg_sv1, v);
+          tc_st8(a_t + (c * 4 + blk) * 8, v);
+        }
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_afull + 8 * t);
+
+      if (!seg_last) continue;
+      // ---------------- epilogue of the segment that ends with this item ----------------
+      const long long tile_begin = tile * a.steps_per_tile;
+      const long long seg_begin = it_begin > tile_begin ? it_begin : tile_begin;
+      const bool complete = (seg_begin == tile_begin) && (step == a.steps_per_tile - 1);
+      const int rt = (int)(tile / a.token_tiles), tt = (int)(tile % a.token_tiles);
+      const int n_out = rt * TILE_ROWS + row;
+      const int m0 = tt * NT;
+      if (!wait_all(bar_accfull, (uint32_t)(seg & 1), 7)) break;
+      tc_fence_after();
+      const int slot_idx = (seg_begin == it_begin) ? 0 : 1;          // first segment of the stripe or not
+      float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(NT * TILE_ROWS);
+#pragma unroll 1
+      for (int c0 = 0; c0 < NT; c0 += 16) {
+        uint32_t v[16];
+        tc_ld16(tmem_base + lane_off + c0, v);
+        tc_wait_ld();
+        if (complete) {
+          if (n_out < a.g.N) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int m = m0 + c0 + j;
+              if (m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * __uint_as_float(v[j]));
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) my_slot[(c0 + j) * TILE_ROWS + row] = __uint_as_float(v[j]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_accempty);
+      ++seg;
+      if (complete) continue;
+      // ---------------- partial tile: publish, count, last arrival reduces ----------------
+      __threadfence();
+      if (!epi_sync()) break;
+      const long long tile_end = tile_begin + a.steps_per_tile;
+      const int c_first = cta_of_item(tile_begin, grid, a.total_items);
+      const int c_last = cta_of_item(tile_end - 1, grid, a.total_items);
+      if (leader) {
+        const uint32_t parts = (uint32_t)(c_last - c_first + 1);
+        const uint32_t prev = atomicAdd(a.counters + tile, 1u);
+        const uint32_t last = (prev + 1 == parts) ? 1u : 0u;
+        if (last) a.counters[tile] = 0;                               // leave the counter ready for the next call
+        __threadfence();
+        *bcast = last;
+      }
+      if (!epi_sync()) break;
+      const bool finisher = *reinterpret_cast<volatile uint32_t*>(bcast) != 0;
+      if (!epi_sync()) break;                                         // bcast may be rewritten after this
+      if (!finisher) continue;
+#pragma unroll 1
+      for (int c0 = 0; c0 < NT; c0 += 16) {
+        float acc[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
+        for (int c = c_first; c <= c_last; ++c) {
+          const long long b_c = (a.total_items * c) / grid;
+          const int sl = (b_c / a.steps_per_tile == tile) ? 0 : 1;
+          const float* src = a.slots + ((size_t)c * 2 + sl) * (size_t)(NT * TILE_ROWS);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) acc[j] += __ldcg(src + (c0 + j) * TILE_ROWS + row);
+        }
+        if (n_out < a.g.N) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            if (m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * acc[j]);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+struct UmmaPlan {
+  int NT, CH;
+  int token_tiles, steps_per_tile, grid;
+  long long tiles, total_items;
+  size_t counters_bytes, slots_bytes;
+};
+
+static UmmaPlan make_plan(const razer_desc* d, int M) {
+  UmmaPlan p;
+  const Geometry g = make_geometry(d->N, d->K);
+  p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
+  p.token_tiles = (M + p.NT - 1) / p.NT;
+  p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
+  p.tiles = (long long)g.row_tiles * p.token_tiles;
+  p.total_items = p.tiles * p.steps_per_tile;
+  const int sms = sm_count();
+  p.grid = (int)(p.total_items < sms ? p.total_items : sms);
+  p.counters_bytes = align256((size_t)p.tiles * sizeof(uint32_t));
+  p.slots_bytes = (size_t)p.grid * 2 * p.NT * TILE_ROWS * sizeof(float);
+  return p;
+}
+
+bool umma_supported(const razer_desc* d, int M) {
+  (void)d;
+  (void)M;
+  // RAZER_KERNEL=simt routes every matmul to the CUDA-core kernel (debugging aid)
+  const char* e = getenv("RAZER_KERNEL");
+  return !(e && e[0] == 's');
+}
+
+size_t umma_workspace_bytes(const razer_desc* d, int M) {
+  // sized for the largest grid (all SMs); the status word comes first
+  UmmaPlan p = make_plan(d, M);
+  const size_t slots = (size_t)(p.grid > 148 ? p.grid : 148) * 2 * p.NT * TILE_ROWS * sizeof(float);
+  return WS_STATUS_BYTES + p.counters_bytes + slots;
+}
+
+template <int NT, int CH, int STAGES, int ASTAGES>
+static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, cudaStream_t st) {
+  using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES>;
+  auto kern = razer_umma_kernel<NT, CH, STAGES, ASTAGES>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES),
+                         "cudaFuncSetAttribute(max dynamic shared memory)"));
+    attr_set = true;
+  }
+  kern<<<grid, UMMA_THREADS, Cfg::SMEM_BYTES, st>>>(tmap, args);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "razer_umma_kernel launch");
+}
+
+int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int M, int ldx_K, float extra_scale,
+                     const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t st) {
+  const Geometry g = make_geometry(d->N, d->K);
+  const UmmaPlan p = make_plan(d, M);
+  const size_t need = WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes;
+  if (!ws || ws_bytes < need)
+    return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)d->K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldx_K * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)CHUNK_K, (cuuint32_t)p.NT};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+
+  UmmaArgs a;
+  a.packed = (const uint8_t*)packed;
+  a.y = (__nv_bfloat16*)y;
+  a.status = (uint32_t*)ws;
+  a.counters = (uint32_t*)((char*)ws + WS_STATUS_BYTES);
+  a.slots = (float*)((char*)ws + WS_STATUS_BYTES + p.counters_bytes);
+  a.extra_scale = extra_scale_dev;
+  a.g = g;
+  a.neg_sv0 = -d->sv_mag[0];
+  a.neg_sv1 = -d->sv_mag[1];
+  a.tensor_scale = d->tensor_scale * extra_scale;
+  a.M = M;
+  a.token_tiles = p.token_tiles;
+  a.steps_per_tile = p.steps_per_tile;
+  a.total_items = p.total_items;
+  switch (p.NT) {
+    case 16: return launch_cfg<16, 4, 6, 2>(tmap, a, p.grid, st);
+    case 32: return launch_cfg<32, 4, 5, 2>(tmap, a, p.grid, st);
+    case 64: return launch_cfg<64, 2, 6, 4>(tmap, a, p.grid, st);
+    case 128: return launch_cfg<128, 1, 8, 4>(tmap, a, p.grid, st);
+    default: return launch_cfg<256, 1, 5, 4>(tmap, a, p.grid, st);
+  }
 }
 
 }  // namespace razer

@@ -65,8 +65,13 @@ def test_dequant_bit_exact_random_codes(b, remap_code, sv_mag):
 # ------------------------------------------------------------------ GEMV / skinny GEMM
 
 def _check_matmul(b, fn, desc, packed, codes, scales, d32, x, rows=None, **kw):
-    y = fn(desc, packed, x.cuda())
-    torch.cuda.synchronize()
+    op = b.OP_GEMV if fn is b.razer_gemv else b.OP_GEMM
+    ws = b.alloc_workspace(desc, x.shape[0], op, "cuda")
+    y = fn(desc, packed, x.cuda(), workspace=ws)
+    b.razer_workspace_status(ws)            # synchronizes; raises if a device wait gave up
+    y2 = fn(desc, packed, x.cuda(), workspace=ws)   # the workspace is left ready for the next call
+    b.razer_workspace_status(ws)
+    assert torch.equal(y, y2), "second call with the same workspace differs"
     xb = inputs.bf16_to_bits(x)
     if rows is None:
         ref = ro.matmul_w4a16(xb, codes, scales, np.float32(d32), **kw)
