@@ -435,6 +435,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
+    __syncwarp();                                       // lane 0 ran the issue loop alone; dealloc is warp-wide
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
                  : "memory");

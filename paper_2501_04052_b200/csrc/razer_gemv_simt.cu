@@ -106,7 +106,8 @@ size_t simt_workspace_bytes(const razer_desc* d, int M) {
   const Geometry g = make_geometry(d->N, d->K);
   const int MT = M >= 8 ? 8 : (M >= 4 ? 4 : (M >= 2 ? 2 : 1));
   const int s = simt_splits(g, M, MT);
-  return s > 1 ? (size_t)s * M * d->N * sizeof(float) : 0;
+  // the first 256 bytes of every workspace hold the device status word
+  return 256 + (s > 1 ? (size_t)s * M * d->N * sizeof(float) : 0);
 }
 
 int launch_gemv_simt(const razer_desc* d, const void* packed, const void* x, int M,
@@ -118,14 +119,15 @@ int launch_gemv_simt(const razer_desc* d, const void* packed, const void* x, int
   int cps = (g.k_chunks + splits - 1) / splits;
   cps = (cps + SIMT_GROUP_CHUNKS - 1) / SIMT_GROUP_CHUNKS * SIMT_GROUP_CHUNKS;
   const int n_splits = (g.k_chunks + cps - 1) / cps;
-  const size_t need = n_splits > 1 ? (size_t)n_splits * M * d->N * sizeof(float) : 0;
+  const size_t need = n_splits > 1 ? 256 + (size_t)n_splits * M * d->N * sizeof(float) : 0;
+  float* partial = ws ? reinterpret_cast<float*>(static_cast<char*>(ws) + 256) : nullptr;
   if (need > ws_bytes || (need && !ws))
     return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
   dim3 grid(g.row_tiles, n_splits, (M + MT - 1) / MT);
   if (grid.z > 65535) return set_error(RAZER_ERR_UNSUPPORTED, "M too large for the CUDA-core kernel");
 #define RAZER_LAUNCH_SIMT(MT_)                                                                      \
   gemv_simt_kernel<MT_><<<grid, TILE_ROWS, 0, st>>>((const uint8_t*)packed, (const __nv_bfloat16*)x, \
-                                                    (__nv_bfloat16*)y, (float*)ws, g, p, extra_scale_dev, M, cps,  \
+                                                    (__nv_bfloat16*)y, partial, g, p, extra_scale_dev, M, cps,  \
                                                     n_splits)
   switch (MT) {
     case 8: RAZER_LAUNCH_SIMT(8); break;
@@ -140,7 +142,7 @@ int launch_gemv_simt(const razer_desc* d, const void* packed, const void* x, int
     const long long mn = (long long)M * d->N;
     long long b = (mn + 255) / 256;
     if (b > 148 * 8) b = 148 * 8;
-    splitk_reduce_kernel<<<(int)b, 256, 0, st>>>((const float*)ws, (__nv_bfloat16*)y, mn, n_splits,
+    splitk_reduce_kernel<<<(int)b, 256, 0, st>>>(partial, (__nv_bfloat16*)y, mn, n_splits,
                                                   d->tensor_scale, extra_scale_dev);
     count_launches(1);
     RAZER_TRY(check_cuda(cudaGetLastError(), "splitk_reduce_kernel launch"));
