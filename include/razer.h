@@ -129,6 +129,27 @@ int razer_gemv_host(const razer_desc* d, const void* packed_dev, const void* x_h
                     void* y_host, void* x_stage_dev, void* y_stage_dev, void* workspace_dev,
                     size_t workspace_bytes, void* stream);
 
+/* razer_gemv for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment convenience of this library).  Some hosts of this code may not call
+ * cudaMalloc: a plug-in running inside another framework's memory pool, a real-time loop
+ * that must not enter the allocator, code running between a stream-capture begin and end.
+ * The other matmul entry points make such callers bring a workspace; this one uses a 4 MiB
+ * scratch array built into the library image instead (every GPU that loads the library holds
+ * those 4 MiB until the process exits), so the caller passes inputs and outputs only.
+ *   1 <= M <= 16.  A shape whose scratch need exceeds the array (tens of millions of rows)
+ *   is rejected with RAZER_ERR_UNSUPPORTED and a message naming both sizes.
+ *   The first call on each device looks up the array's device address (with that device
+ *   current); make that first call outside any stream capture.  No call allocates or frees.
+ *   All calls on one device share the array and it keeps the previous call's contents; the
+ *   entry point clears the part that must start at zero on `stream` before the kernel.  Two
+ *   calls that can overlap on the GPU (different streams without an ordering between them)
+ *   would race on it: order them, or use razer_gemv with separate workspaces.
+ *   A device-side wait that gives up leaves y undefined; it is not reported by this entry
+ *   point (there is no workspace to query) - use razer_gemv where that matters.
+ * Result and argument meaning are those of razer_gemv. */
+int razer_gemv_static(const razer_desc* d, const void* packed_dev, const void* x_dev, int M,
+                      void* y_dev, void* stream);
+
 /* Online activation quantization (Sec. 4.2: each block is quantized once per allowed
  * special value, +sv_mag and -sv_mag, and the lower squared error wins; Eq. 1-3, 6-7 with
  * the 7-bit E4M3 block scale).  x_dev: bf16 [M][K], K multiple of 16.

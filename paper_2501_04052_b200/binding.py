@@ -24,7 +24,7 @@ OP_GEMV, OP_GEMM, OP_GEMM_W4A4 = 0, 1, 2
 EXPORTS = (
     "razer_last_error", "razer_version", "razer_kernel_launches", "razer_packed_bytes", "razer_pack_layout", "razer_dequant",
     "razer_workspace_bytes", "razer_workspace_init", "razer_workspace_status", "razer_gemv", "razer_gemm", "razer_gemv_host", "razer_quant_act",
-    "razer_decode_act", "razer_gemm_w4a4",
+    "razer_decode_act", "razer_gemm_w4a4", "razer_gemv_static",
 )
 
 
@@ -58,6 +58,7 @@ _lib.razer_gemv.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_voi
 _lib.razer_gemm.argtypes = _lib.razer_gemv.argtypes
 _lib.razer_gemv_host.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                  c_void_p, c_size_t, c_void_p]
+_lib.razer_gemv_static.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_void_p, c_void_p]
 _lib.razer_quant_act.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p, c_void_p,
                                  c_void_p, c_void_p]
 _lib.razer_decode_act.argtypes = [c_void_p, c_void_p, c_int, c_int, c_float, c_void_p, c_void_p]
@@ -172,6 +173,15 @@ def razer_gemv(desc, packed, x, y=None, workspace=None) -> torch.Tensor:
 def razer_gemm(desc, packed, x, y=None, workspace=None) -> torch.Tensor:
     """x bf16 [M, K] (device) -> y bf16 [M, N]."""
     return _matmul(_lib.razer_gemm, desc, packed, x, y, workspace, OP_GEMM)
+
+
+def razer_gemv_static(desc, packed, x, y) -> torch.Tensor:
+    """razer_gemv without a workspace argument: the library's built-in scratch array is used, so
+    nothing is allocated here either (the caller brings y).  x bf16 [M, K] with M <= 16."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.shape[1] == desc.K
+    assert y.is_cuda and y.dtype == torch.bfloat16 and y.is_contiguous() and tuple(y.shape) == (x.shape[0], desc.N)
+    _check(_lib.razer_gemv_static(ctypes.byref(desc), _ptr(packed), _ptr(x), x.shape[0], _ptr(y), _stream()))
+    return y
 
 
 def razer_gemv_host(desc, packed, x_host, y_host, x_stage, y_stage, workspace) -> None:

@@ -509,6 +509,11 @@ size_t umma_workspace_bytes(const razer_desc* d, int M) {
   return WS_STATUS_BYTES + p.counters_bytes + slots;
 }
 
+// Leading part of the workspace that has to be zero before a launch (status word + counters).
+size_t umma_workspace_zero_bytes(const razer_desc* d, int M) {
+  return WS_STATUS_BYTES + make_plan(d, M).counters_bytes;
+}
+
 template <int NT, int CH, int STAGES, int ASTAGES>
 static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, cudaStream_t st) {
   using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES>;
