@@ -16,19 +16,25 @@ namespace razer {
 //
 // The tensor is cut into tiles of TILE_ROWS rows x CHUNK_K columns (4 blocks of 16).
 // One tile-chunk is CHUNK_BYTES contiguous bytes:
-//   [blk 0..3][row 0..127] 8 bytes : the block's 16 nibbles, element j of the block in
-//                                    nibble j (byte j/2, low nibble first)
+//   [blk 0..3][row 0..127] 8 bytes : the block's 16 nibbles as two 32-bit words; element j of
+//                                    the block sits in word j/8, nibble (j%8)/2 + 4*(j%2), so
+//                                    that nibbles p and p+4 of a word (the same position in
+//                                    its two 16-bit halves) are elements 2p and 2p+1
 //   [row 0..127] 4 bytes           : the four blocks' scale bytes
 // so that thread = row reads are contiguous across a warp (8 B or 4 B stride) and a whole
 // chunk is one bulk copy.  Chunks are ordered [row tile][k chunk].  Rows beyond N and
 // columns beyond K are zero blocks (scale byte 0).
 //
 // Inside the packed form:
-//   * the special value is always code 0x8, a true zero always code 0x0;
-//   * a block whose special value is positive is stored negated (sign bits of all non-zero
-//     codes flipped) so that code 0x8 always means "-sv_mag[select]";
+//   * the special value is always nibble 0x0, a true zero always nibble 0x8, every other
+//     nibble is S E1 E0 M as in Eq. 5;
+//   * a block whose special value is negative is stored negated (sign bits of all non-zero
+//     codes flipped) so that nibble 0x0 always means "+sv_mag[select]";
 //   * scale byte = [negate | select | 6-bit scale code]; negate = 1 means the block's
 //     values are the negatives of the stored codes' values.
+// With these conventions the decoder needs no comparison: the nibble's bits drop into a
+// bf16 bit pattern (sign to bit 15, E1 E0 M to bits 8:6, value x 2^-126), the special value
+// is the one nibble that is numerically zero, and the block sign rides on the scale.
 // ---------------------------------------------------------------------------------
 constexpr int TILE_ROWS = 128;
 constexpr int CHUNK_K = 64;
@@ -98,11 +104,22 @@ __device__ __forceinline__ float scale_value(uint32_t code) {
   return e ? normal : (float)m * 0.001953125f;   // m * 2^-9
 }
 
-// Element value of a packed-form nibble: code 0x8 is -sv, everything else Eq. 5.
-__device__ __forceinline__ float packed_elem(uint32_t nib, float neg_sv) {
+// Position (in bits) of element j's nibble inside the block's 64-bit code word.
+__host__ __device__ __forceinline__ int packed_nibble_shift(int j) {
+  return 32 * (j >> 3) + 4 * (((j & 7) >> 1) + 4 * (j & 1));
+}
+
+// Stored nibble of element j of a packed block.
+__device__ __forceinline__ uint32_t packed_nibble(uint2 cw, int j) {
+  const int sh = packed_nibble_shift(j);
+  return ((sh < 32 ? cw.x >> sh : cw.y >> (sh - 32))) & 0xFu;
+}
+
+// Element value of a packed-form nibble: 0x0 is +sv, 0x8 is zero, everything else Eq. 5.
+__device__ __forceinline__ float packed_elem(uint32_t nib, float sv) {
   const float mag = fp4_mag(nib & 7u);
   const float v = (nib & 8u) ? -mag : mag;
-  return (nib == 8u) ? neg_sv : v;
+  return (nib == 0u) ? sv : v;
 }
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b) {

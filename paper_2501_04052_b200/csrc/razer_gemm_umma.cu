@@ -6,12 +6,21 @@
 // (128 weight rows = 128 TMEM lanes), the activation tile is the B operand (NT tokens,
 // K-major in shared memory, 128-byte swizzle, written by TMA), the accumulator D[128 x NT]
 // lives in TMEM.  Weights never exist as bf16 in shared or global memory: a TMA bulk copy
-// brings the packed 4.5-bit chunk into shared memory, four "dequant" warps (thread = weight
+// brings the packed 4.5-bit chunk into shared memory, the "dequant" warps (thread = weight
 // row) decode one 16-element block at a time in registers and write the bf16 pairs straight
 // into TMEM with tcgen05.st, and the MMA reads A from TMEM.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
-// warps 2..5 = dequant, then epilogue of the tile they just fed.
+// Warp roles (64 + 32 * NDW threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA
+// issuer, warps 2.. = dequant.  A warp reaches only the TMEM lanes 32 * (warp % 4) .. + 31, so
+// warps w and w + 4 own the same 32 weight rows and split the stage's blocks between them;
+// the first four dequant warps also run the epilogue of the tile they just fed.
+//
+// Decode (per pair of elements, no comparison, no conversion instruction): the stored nibble
+// is isolated in both 16-bit halves of the word, one integer multiply-add drops two shifted
+// copies of it, one logic op keeps sign -> bit 15 and E1 E0 M -> bits 8:6 (a bf16 pattern worth
+// value x 2^-126, subnormal for 0.5) and ORs in the special value, which one fused
+// multiply-add with ReLU derives from the isolated nibble (it is the only nibble that is
+// numerically zero); one packed bf16 multiply by +-scale x 2^126 finishes the exact product.
 //
 // Work partition (Sec. 4.3 / App. E of the paper: stripes of about equal length that may span
 // several output tiles, partial results reduced through global memory): the grid is
@@ -32,7 +41,8 @@ namespace razer {
 
 // ------------------------------------------------------------------ workspace layout
 constexpr size_t WS_STATUS_BYTES = 256;               // word 0: device status (0 = ok)
-constexpr int UMMA_THREADS = 192;
+constexpr int NDW = 8;                                // dequant warps (a multiple of 4)
+constexpr int UMMA_THREADS = 64 + 32 * NDW;
 constexpr uint32_t WAIT_LIMIT = 1u << 26;             // try_wait rounds before giving up, and
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;     // wall-clock bound of one wait (2 s)
 
@@ -140,22 +150,47 @@ __host__ __device__ constexpr uint32_t make_idesc(int nt) {
 }
 
 // ------------------------------------------------------------------ decode (registers)
-// One packed block (16 nibbles + scale byte) -> 8 registers of two bf16 each, element 2p in
-// the low half of register p.  block_scale * element has at most 8 significant bits, so the
-// FP32 product's upper 16 bits are the exact bf16.
-__device__ __forceinline__ void decode_block_bf16(uint2 cw, uint32_t sb, float neg_sv0, float neg_sv1,
-                                                  uint32_t (&out)[8]) {
-  float s = scale_value(sb & 0x3Fu);
-  if (sb & 0x80u) s = -s;
-  const float neg_sv = (sb & 0x40u) ? neg_sv1 : neg_sv0;
-#pragma unroll
-  for (int p = 0; p < 8; ++p) {
-    const uint32_t w = (p < 4) ? cw.x : cw.y;
-    const uint32_t byte = (w >> (8 * (p & 3))) & 0xFFu;
-    const float a = packed_elem(byte & 0xFu, neg_sv) * s;
-    const float b = packed_elem(byte >> 4, neg_sv) * s;
-    out[p] = (__float_as_uint(a) >> 16) | (__float_as_uint(b) & 0xFFFF0000u);
-  }
+__device__ __forceinline__ uint32_t fma_relu_bf16x2(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.relu.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
+// Per-block decode constants, looked up in shared memory by the block's scale byte.
+struct SvConsts {            // indexed by the select bit
+  uint32_t sv;               // (sv, sv) x 2^-126 as bf16x2
+  uint32_t nsv_lo;           // -(sv x 2^7):  sv_pattern - nsv_lo * (nibble in bits 3:0 read as bf16) = 0 for nibble 1
+  uint32_t nsv_hi;           // -(sv x 2^3):  the same for a nibble in bits 7:4
+  uint32_t pad;
+};
+
+// Four stored nibbles of each 16-bit half of `w` -> four bf16x2 registers (elements 2p, 2p+1
+// of the word in register p), each the exact product value x scale with the block's sign.
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t ss2, const SvConsts& c, uint32_t mul_lo,
+                                            uint32_t mul_hi, uint32_t* out) {
+  const uint32_t w8 = w >> 8;
+  const uint32_t n0 = w & 0x000F000Fu, n1 = w & 0x00F000F0u;
+  const uint32_t n2 = w8 & 0x000F000Fu, n3 = w8 & 0x00F000F0u;
+  // nibble * (2^6 + 2^12) [bits 3:0] or * (2^2 + 2^8) [bits 7:4]: one copy lands with E1 E0 M on
+  // bits 8:6, the other with S on bit 15; the mask keeps exactly those
+  const uint32_t u0 = and_or(n0 * mul_lo, 0x81C081C0u, fma_relu_bf16x2(n0, c.nsv_lo, c.sv));
+  const uint32_t u1 = and_or(n1 * mul_hi, 0x81C081C0u, fma_relu_bf16x2(n1, c.nsv_hi, c.sv));
+  const uint32_t u2 = and_or(n2 * mul_lo, 0x81C081C0u, fma_relu_bf16x2(n2, c.nsv_lo, c.sv));
+  const uint32_t u3 = and_or(n3 * mul_hi, 0x81C081C0u, fma_relu_bf16x2(n3, c.nsv_hi, c.sv));
+  out[0] = mul_bf16x2(u0, ss2);
+  out[1] = mul_bf16x2(u1, ss2);
+  out[2] = mul_bf16x2(u2, ss2);
+  out[3] = mul_bf16x2(u3, ss2);
 }
 
 // ------------------------------------------------------------------ kernel
@@ -167,7 +202,8 @@ struct UmmaArgs {
   uint32_t* status;          // device status word
   const float* extra_scale;  // optional device scalar multiplied into the tensor scale
   Geometry g;
-  float neg_sv0, neg_sv1, tensor_scale;
+  float sv0, sv1, tensor_scale;
+  uint32_t mul_lo, mul_hi;   // 2^6 + 2^12 and 2^2 + 2^8, passed at run time so that they stay multiplies
   int M, token_tiles, steps_per_tile;
   long long total_items;
 };
@@ -185,7 +221,9 @@ struct UmmaCfg {
   static constexpr int TMEM_COLS = TMEM_COLS_NEEDED <= 64 ? 64 : TMEM_COLS_NEEDED <= 128 ? 128
                                    : TMEM_COLS_NEEDED <= 256 ? 256 : 512;
   static constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 3;
-  static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + NUM_BARS * 8 + 64;
+  static constexpr int TABLE_BYTES = 256 * 4 + 2 * 16;         // scale-byte table + special-value constants
+  static constexpr size_t SMEM_BYTES =
+      1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + NUM_BARS * 8 + 16 + 64 + TABLE_BYTES;
   static_assert(TMEM_COLS_NEEDED <= 512, "TMEM budget exceeded");
   static_assert(NT % 16 == 0 && NT >= 16 && NT <= 256, "UMMA N for M = 128");
 };
@@ -201,9 +239,12 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * Cfg::STAGE_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + Cfg::NUM_BARS);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(        // 16-byte aligned: the tables behind it are read as uint4
+      (reinterpret_cast<uintptr_t>(bars + Cfg::NUM_BARS) + 15) & ~(uintptr_t)15);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   uint32_t* bcast = tmem_slot + 2;                      // epilogue broadcast word
+  uint32_t* ss_tab = tmem_slot + 16;                    // [256] (+-scale x 2^126) as bf16x2, by scale byte
+  SvConsts* sv_tab = reinterpret_cast<SvConsts*>(ss_tab + 256);   // [2] by select bit
 
   const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> dequant, MMA
   const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]  MMA commit -> TMA
@@ -224,7 +265,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       mbar_init(bar_empty + 8 * i, 1);
     }
     for (int i = 0; i < ASTAGES; ++i) {
-      mbar_init(bar_afull + 8 * i, 128);
+      mbar_init(bar_afull + 8 * i, 32 * NDW);
       mbar_init(bar_aempty + 8 * i, 1);
     }
     mbar_init(bar_accfull, 1);
@@ -233,6 +274,24 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     *abort_flag = 0;
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = threadIdx.x; i < 256; i += UMMA_THREADS) {
+    // scale x 2^126 has four significant bits: the upper half of the FP32 pattern is the exact bf16
+    const float sc = scale_value((uint32_t)i & 0x3Fu) * 8.50705917e37f;   // 2^126
+    const uint32_t b = (__float_as_uint(sc) >> 16) | (((uint32_t)i & 0x80u) << 8);
+    ss_tab[i] = b | (b << 16);
+  }
+  if (threadIdx.x < 2) {
+    const float sv = threadIdx.x ? a.sv1 : a.sv0;          // at most four significant bits
+    const uint32_t p0 = __float_as_uint(sv * 1.17549435e-38f) >> 16;     // sv x 2^-126
+    const uint32_t p1 = __float_as_uint(-sv * 128.0f) >> 16;
+    const uint32_t p2 = __float_as_uint(-sv * 8.0f) >> 16;
+    SvConsts c;
+    c.sv = p0 | (p0 << 16);
+    c.nsv_lo = p1 | (p1 << 16);
+    c.nsv_hi = p2 | (p2 << 16);
+    c.pad = 0;
+    sv_tab[threadIdx.x] = c;
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -311,9 +370,12 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       }
     }
   } else {
-    // ===================== dequant + epilogue (128 threads, thread = weight row) =====================
+    // ===================== dequant (32 * NDW threads, thread = weight row) + epilogue =====================
     const int row = 32 * (warp & 3) + lane;              // TMEM lane this thread owns
     const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
+    const int sub = (warp - 2) >> 2;                     // which share of a stage's blocks this warp decodes
+    constexpr int SUBS = NDW / 4;
+    const bool epi_warp = (sub == 0);                    // warps 2..5 also run the epilogue
     const bool leader = (threadIdx.x == 64);
     const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
     long long n = 0, seg = 0;
@@ -330,6 +392,8 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       ++epi_phase;
       return got;
     };
+    const uint8_t* ss_bytes = reinterpret_cast<const uint8_t*>(ss_tab);
+    const uint8_t* sv_bytes = reinterpret_cast<const uint8_t*>(sv_tab);
     for (long long it = it_begin; it < it_end; ++it, ++n) {
       const int s = (int)(n % STAGES), t = (int)(n % ASTAGES);
       const uint32_t ph = (uint32_t)((n / STAGES) & 1), aph = (uint32_t)((n / ASTAGES) & 1);
@@ -346,10 +410,17 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         const uint8_t* ck = st + c * CHUNK_BYTES;
         const uint32_t sw = *reinterpret_cast<const uint32_t*>(ck + CHUNK_CODE_BYTES + row * 4);
 #pragma unroll
-        for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
+        for (int bq = 0; bq < CHUNK_BLOCKS / SUBS; ++bq) {
+          const int blk = bq * SUBS + sub;
           const uint2 cw = *reinterpret_cast<const uint2*>(ck + (blk * TILE_ROWS + row) * 8);
+          // byte offsets into the two tables, straight from the scale word
+          const uint32_t off_ss = (blk == 0 ? sw << 2 : sw >> (8 * blk - 2)) & 0x3FCu;
+          const uint32_t off_sv = (sw >> (8 * blk + 2)) & 0x10u;
+          const uint32_t ss2 = *reinterpret_cast<const uint32_t*>(ss_bytes + off_ss);
+          const SvConsts svc = *reinterpret_cast<const SvConsts*>(sv_bytes + off_sv);
           uint32_t v[8];
-          decode_block_bf16(cw, (sw >> (8 * blk)) & 0xFFu, a.neg_sv0, a.neg_sv1, v);
+          decode_word(cw.x, ss2, svc, a.mul_lo, a.mul_hi, v);
+          decode_word(cw.y, ss2, svc, a.mul_lo, a.mul_hi, v + 4);
           tc_st8(a_t + (c * 4 + blk) * 8, v);
         }
       }
@@ -357,7 +428,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       tc_fence_before();
       mbar_arrive(bar_afull + 8 * t);
 
-      if (!seg_last) continue;
+      if (!seg_last || !epi_warp) continue;
       // ---------------- epilogue of the segment that ends with this item ----------------
       const long long tile_begin = tile * a.steps_per_tile;
       const long long seg_begin = it_begin > tile_begin ? it_begin : tile_begin;
@@ -556,8 +627,10 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   a.slots = (float*)((char*)ws + WS_STATUS_BYTES + p.counters_bytes);
   a.extra_scale = extra_scale_dev;
   a.g = g;
-  a.neg_sv0 = -d->sv_mag[0];
-  a.neg_sv1 = -d->sv_mag[1];
+  a.sv0 = d->sv_mag[0];
+  a.sv1 = d->sv_mag[1];
+  a.mul_lo = (1u << 6) + (1u << 12);
+  a.mul_hi = (1u << 2) + (1u << 8);
   a.tensor_scale = d->tensor_scale * extra_scale;
   a.M = M;
   a.token_tiles = p.token_tiles;

@@ -21,7 +21,7 @@ gemv_simt_kernel(const uint8_t* __restrict__ packed, const __nv_bfloat16* __rest
   const int row_in = threadIdx.x;
   const int c_begin = split * chunks_per_split;
   const int c_end = min(g.k_chunks, c_begin + chunks_per_split);
-  const float neg_sv0 = -p.sv_mag[0], neg_sv1 = -p.sv_mag[1];
+  const float sv0 = p.sv_mag[0], sv1 = p.sv_mag[1];
   float acc[MT];
 #pragma unroll
   for (int m = 0; m < MT; ++m) acc[m] = 0.0f;
@@ -46,15 +46,14 @@ gemv_simt_kernel(const uint8_t* __restrict__ packed, const __nv_bfloat16* __rest
         const uint32_t sb = (sw >> (8 * blk)) & 0xFFu;
         float s = scale_value(sb & 0x3Fu);
         if (sb & 0x80u) s = -s;
-        const float neg_sv = (sb & 0x40u) ? neg_sv1 : neg_sv0;
+        const float sv = (sb & 0x40u) ? sv1 : sv0;
         float part[MT];
 #pragma unroll
         for (int m = 0; m < MT; ++m) part[m] = 0.0f;
         const int kk0 = (c - cg) * CHUNK_K + blk * 16;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const uint32_t w = (j < 8) ? cw.x : cw.y;
-          const float q = packed_elem((w >> (4 * (j & 7))) & 0xFu, neg_sv);
+          const float q = packed_elem(packed_nibble(cw, j), sv);
 #pragma unroll
           for (int m = 0; m < MT; ++m) part[m] = fmaf(q, xs[m][kk0 + j], part[m]);
         }

@@ -24,25 +24,30 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __
       w1 = c.y;
       sb = scales[(size_t)n * (g.K / 16) + kb];
     }
-    // nibble-wise masks: has_mag = low three bits non-zero, replicated to the sign position
+    // bit 3 of each nibble of nz is set iff the nibble's magnitude (low three bits) is non-zero
     auto canon = [&](uint32_t w, bool negate) -> uint32_t {
       const uint32_t m = w & 0x77777777u;
-      // bit 3 of each nibble set iff the nibble's magnitude is non-zero
       const uint32_t nz = ((m + 0x77777777u) & 0x88888888u);
-      if (remap_code == 0) w ^= (~nz) & 0x88888888u;   // swap the two zero codes
+      if (remap_code == 0x8) w ^= (~nz) & 0x88888888u;  // packed form: special value 0x0, true zero 0x8
       if (negate) w ^= nz;                              // flip the sign of non-zero codes
       return w;
     };
+    // interchange nibble order (element j in nibble j) -> packed order (nibbles p and p+4 = elements 2p, 2p+1)
+    auto shuffle = [](uint32_t w) -> uint32_t {
+      uint32_t o = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o |= ((w >> (4 * j)) & 0xFu) << (4 * ((j >> 1) + 4 * (j & 1)));
+      return o;
+    };
     const uint32_t scode = sb & 0x3Fu;
-    const bool sv_negative = (sb & 0x80u) != 0;
-    const bool negate = !sv_negative;
+    const bool negate = (sb & 0x80u) != 0;              // negative special value: store the block negated
     uint32_t out_sb = 0;
     if (scode != 0) {
       out_sb = (negate ? 0x80u : 0u) | (sb & 0x40u) | scode;
-      w0 = canon(w0, negate);
-      w1 = canon(w1, negate);
+      w0 = shuffle(canon(w0, negate));
+      w1 = shuffle(canon(w1, negate));
     } else {
-      w0 = w1 = 0;                                      // zero block: nothing to keep
+      w0 = w1 = 0x88888888u;                            // zero block: sixteen true zeros
     }
     uint8_t* base = packed + (size_t)chunk * CHUNK_BYTES;
     *reinterpret_cast<uint2*>(base + ((size_t)blk * TILE_ROWS + row_in) * 8) = make_uint2(w0, w1);
@@ -71,12 +76,10 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ packed, void* __restr
     const uint32_t sb = base[CHUNK_CODE_BYTES + row_in * 4 + blk];
     float s = scale_value(sb & 0x3Fu);
     if (sb & 0x80u) s = -s;
-    const float neg_sv = -p.sv_mag[(sb >> 6) & 1u];
+    const float sv = p.sv_mag[(sb >> 6) & 1u];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const uint32_t w = (j < 8) ? c.x : c.y;
-      const uint32_t nib = (w >> (4 * (j & 7))) & 0xFu;
-      float d1 = packed_elem(nib, neg_sv) * s;        // exact: <= 8 significant bits
+      float d1 = packed_elem(packed_nibble(c, j), sv) * s;   // exact: <= 8 significant bits
       d1 = __fadd_rn(d1, 0.0f);                       // canonical +0 (-0 + 0 = +0)
       const size_t o = (size_t)n * g.K + k0 + j;
       if (FP32_OUT) {
