@@ -14,7 +14,7 @@ from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_size_t, c_void_
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librazer.so")
+LIB_PATH = os.environ.get("RAZER_LIB") or os.path.join(_HERE, "librazer.so")   # RAZER_LIB: load another build of the library
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = -1, -2, -3, -4, -5

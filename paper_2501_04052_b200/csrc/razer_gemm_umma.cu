@@ -41,8 +41,6 @@ namespace razer {
 
 // ------------------------------------------------------------------ workspace layout
 constexpr size_t WS_STATUS_BYTES = 256;               // word 0: device status (0 = ok)
-constexpr int NDW = 8;                                // dequant warps (a multiple of 4)
-constexpr int UMMA_THREADS = 64 + 32 * NDW;
 constexpr uint32_t WAIT_LIMIT = 1u << 26;             // try_wait rounds before giving up, and
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;     // wall-clock bound of one wait (2 s)
 
@@ -101,6 +99,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+// True in exactly one lane of a converged warp.  Loops that only issue asynchronous work run
+// on the whole warp with this predicate around the issuing instructions, so that addresses
+// and descriptors stay warp-uniform values.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -114,6 +126,19 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Same with the shared-memory descriptor given as two 32-bit halves (only the low half changes
+// from one MMA to the next) and the accumulate flag known at compile time.
+template <bool ACCUMULATE>
+__device__ __forceinline__ void tc_mma_ts2(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_desc_lo, uint32_t b_desc_hi,
+                                           uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 bd, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "n"(ACCUMULATE ? 1 : 0)
       : "memory");
 }
 __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
@@ -205,17 +230,18 @@ struct UmmaArgs {
   float sv0, sv1, tensor_scale;
   uint32_t mul_lo, mul_hi;   // 2^6 + 2^12 and 2^2 + 2^8, passed at run time so that they stay multiplies
   int M, token_tiles, steps_per_tile;
+  int x_map_3d;              // the activation tensor map is the 3-D (64 k, tokens, k chunk) view: one load per stage
   long long total_items;
 };
 
-template <int NT, int CH, int STAGES, int ASTAGES>
+template <int NT, int CH, int STAGES, int ASTAGES, int NACC>
 struct UmmaCfg {
   static constexpr int W_BYTES = CH * CHUNK_BYTES;
   static constexpr int X_BOX_BYTES = NT * 128;                 // NT tokens x 64 k x 2 B
   static constexpr int X_BYTES = CH * X_BOX_BYTES;
   static constexpr int W_PAD = (W_BYTES + 1023) / 1024 * 1024; // keep the x boxes 1024-byte aligned
   static constexpr int STAGE_BYTES = W_PAD + X_BYTES;
-  static constexpr int ACC_COLS = NT < 32 ? 32 : NT;
+  static constexpr int ACC_COLS = NACC * NT < 32 ? 32 : NACC * NT;   // NACC accumulators, used round robin
   static constexpr int A_STAGE_COLS = CH * 32;                 // 4 blocks x 8 columns per chunk
   static constexpr int TMEM_COLS_NEEDED = ACC_COLS + ASTAGES * A_STAGE_COLS;
   static constexpr int TMEM_COLS = TMEM_COLS_NEEDED <= 64 ? 64 : TMEM_COLS_NEEDED <= 128 ? 128
@@ -232,10 +258,25 @@ __device__ __forceinline__ int cta_of_item(long long item, int grid, long long t
   return (int)((((item + 1) * grid) - 1) / total);
 }
 
-template <int NT, int CH, int STAGES, int ASTAGES>
-__global__ void __launch_bounds__(UMMA_THREADS, 1)
+// Position of a CTA inside its stripe of work items; advanced one item at a time so that
+// the hot loops need no division.
+struct ItemCursor {
+  int tile, step;          // output tile and k-stage inside it
+  int stage, phase;        // ring slot of the shared-memory stage and its parity
+  int astage, aphase;      // ring slot of the TMEM A stage and its parity
+  template <int STAGES, int ASTAGES>
+  __device__ __forceinline__ void next(int steps_per_tile) {
+    if (++step == steps_per_tile) { step = 0; ++tile; }
+    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+    if (++astage == ASTAGES) { astage = 0; aphase ^= 1; }
+  }
+};
+
+template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC>
+__global__ void __launch_bounds__(64 + 32 * NDW, 1)
 razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) {
-  using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES>;
+  using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES, NACC>;
+  constexpr int THREADS = 64 + 32 * NDW;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * Cfg::STAGE_BYTES);
@@ -256,8 +297,14 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grid = gridDim.x, cta = blockIdx.x;
-  const long long it_begin = (a.total_items * cta) / grid;
-  const long long it_end = (a.total_items * (cta + 1)) / grid;
+  const int it_begin = (int)((a.total_items * cta) / grid);
+  const int it_end = (int)((a.total_items * (cta + 1)) / grid);
+  const int n_items = it_end - it_begin;
+  const int spt = a.steps_per_tile;
+  ItemCursor cur;
+  cur.tile = it_begin / spt;
+  cur.step = it_begin - cur.tile * spt;
+  cur.stage = cur.phase = cur.astage = cur.aphase = 0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
@@ -265,7 +312,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       mbar_init(bar_empty + 8 * i, 1);
     }
     for (int i = 0; i < ASTAGES; ++i) {
-      mbar_init(bar_afull + 8 * i, 32 * NDW);
+      mbar_init(bar_afull + 8 * i, 128);
       mbar_init(bar_aempty + 8 * i, 1);
     }
     mbar_init(bar_accfull, 1);
@@ -275,7 +322,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = threadIdx.x; i < 256; i += UMMA_THREADS) {
+  for (int i = threadIdx.x; i < 256; i += THREADS) {
     // scale x 2^126 has four significant bits: the upper half of the FP32 pattern is the exact bf16
     const float sc = scale_value((uint32_t)i & 0x3Fu) * 8.50705917e37f;   // 2^126
     const uint32_t b = (__float_as_uint(sc) >> 16) | (((uint32_t)i & 0x80u) << 8);
@@ -314,72 +361,87 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     // ===================== TMA producer =====================
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
-      long long issued = 0;
-      for (long long it = it_begin; it < it_end; ++it, ++issued) {
-        const int s = (int)(issued % STAGES);
-        const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
-        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { fail(1); break; }
-        const long long tile = it / a.steps_per_tile;
-        const int step = (int)(it % a.steps_per_tile);
-        const int rt = (int)(tile / a.token_tiles), tt = (int)(tile % a.token_tiles);
-        const int c0 = step * CH;
+      int issued = 0;
+      int rt = cur.tile / a.token_tiles, tt = cur.tile - rt * a.token_tiles;
+      for (; issued < n_items; ++issued) {
+        if (!mbar_wait(bar_empty + 8 * cur.stage, (uint32_t)cur.phase ^ 1u, abort_flag)) { fail(1); break; }
+        const int c0 = cur.step * CH;
         const int nch = min(CH, a.g.k_chunks - c0);
-        uint8_t* st = smem + (size_t)s * Cfg::STAGE_BYTES;
-        mbar_expect_tx(bar_full + 8 * s, (uint32_t)(nch * (CHUNK_BYTES + Cfg::X_BOX_BYTES)));
-        bulk_copy_g2s(smem_u32(st), a.packed + ((size_t)rt * a.g.k_chunks + c0) * CHUNK_BYTES,
-                      (uint32_t)(nch * CHUNK_BYTES), bar_full + 8 * s);
-        for (int c = 0; c < nch; ++c)
-          tma_load_2d(smem_u32(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES), &tmap_x, (c0 + c) * CHUNK_K, tt * NT,
-                      bar_full + 8 * s);
+        const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
+        const uint32_t bar = bar_full + 8 * cur.stage;
+        const uint32_t n_x = a.x_map_3d ? CH : nch;       // the 3-D box always spans CH chunks (zero-filled past K)
+        mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * Cfg::X_BOX_BYTES);
+        bulk_copy_g2s(st, a.packed + ((size_t)rt * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
+        if (a.x_map_3d) {
+          tma_load_3d(st + Cfg::W_PAD, &tmap_x, 0, tt * NT, c0, bar);
+        } else {
+          for (int c = 0; c < nch; ++c)
+            tma_load_2d(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, tt * NT, bar);
+        }
+        if (cur.step == spt - 1 && ++tt == a.token_tiles) { tt = 0; ++rt; }
+        cur.template next<STAGES, ASTAGES>(spt);
       }
       // Drain: copies still in flight must land before this CTA's shared memory is released.
-      const long long pending = issued < STAGES ? issued : STAGES;
-      for (long long f = issued - pending; f < issued; ++f)
-        mbar_wait(bar_full + 8 * (int)(f % STAGES), (uint32_t)((f / STAGES) & 1), tmem_slot + 3);
+      const int pending = issued < STAGES ? issued : STAGES;
+      for (int f = issued - pending; f < issued; ++f)
+        mbar_wait(bar_full + 8 * (f % STAGES), (uint32_t)((f / STAGES) & 1), tmem_slot + 3);
     }
   } else if (warp == 1) {
-    // ===================== MMA issuer =====================
-    if (lane == 0) {
+    // ===================== MMA issuer (whole warp walks the items, one elected lane issues) =====================
+    {
       constexpr uint32_t idesc = make_idesc(NT);
-      long long n = 0, seg = 0;
-      for (long long it = it_begin; it < it_end; ++it, ++n) {
-        const int s = (int)(n % STAGES), t = (int)(n % ASTAGES);
-        const uint32_t ph = (uint32_t)((n / STAGES) & 1), aph = (uint32_t)((n / ASTAGES) & 1);
-        const long long tile = it / a.steps_per_tile;
-        const int step = (int)(it % a.steps_per_tile);
-        const bool seg_first = (it == it_begin) || step == 0;
-        const bool seg_last = (it + 1 == it_end) || step == a.steps_per_tile - 1;
-        const int nch = min(CH, a.g.k_chunks - step * CH);
-        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { fail(2); break; }
-        if (!mbar_wait(bar_afull + 8 * t, aph, abort_flag)) { fail(3); break; }
-        if (seg_first && !mbar_wait(bar_accempty, (uint32_t)((seg & 1) ^ 1), abort_flag)) { fail(4); break; }
+      // upper half of the shared-memory descriptor: 1024-byte group stride, descriptor version, 128-byte swizzle
+      constexpr uint32_t bd_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      uint32_t seg = 0;
+      auto wait_warp = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
+        const bool got = mbar_wait(bar, parity, abort_flag);
+        if (!got) fail(code);
+        return __all_sync(0xFFFFFFFFu, got);
+      };
+      for (int i = 0; i < n_items; ++i) {
+        const bool seg_first = (i == 0) || cur.step == 0;
+        const bool seg_last = (i + 1 == n_items) || cur.step == spt - 1;
+        const int nch = min(CH, a.g.k_chunks - cur.step * CH);
+        if (!wait_warp(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 2)) break;
+        if (!wait_warp(bar_afull + 8 * cur.astage, (uint32_t)cur.aphase, 3)) break;
+        if (seg_first && !wait_warp(bar_accempty, (seg & 1u) ^ 1u, 4)) break;
         tc_fence_after();
-        const uint32_t xs = smem_u32(smem + (size_t)s * Cfg::STAGE_BYTES + Cfg::W_PAD);
-        const uint32_t a_t = tmem_a0 + t * Cfg::A_STAGE_COLS;
-        for (int j = 0; j < nch * 4; ++j) {
-          const uint64_t bd = make_b_desc(xs + (j >> 2) * Cfg::X_BOX_BYTES + (j & 3) * 32);
-          tc_mma_ts(tmem_base, a_t + j * 8, bd, idesc, (seg_first && j == 0) ? 0u : 1u);
+        const uint32_t xs = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES + Cfg::W_PAD;
+        const uint32_t a_t = tmem_a0 + cur.astage * Cfg::A_STAGE_COLS;
+        const uint32_t bd_lo = (xs >> 4) | (1u << 16);    // start address and (unused) leading offset fields
+        if (elect_one()) {
+          // Consecutive MMAs go to NACC different accumulators (summed in the epilogue): MMAs on one
+          // accumulator execute one after the other, and a narrow MMA is far shorter than its latency.
+#pragma unroll
+          for (int j = 0; j < CH * 4; ++j) {
+            // 16 k further along: +32 bytes inside a chunk's 128-byte rows, next chunk's box after four
+            if (j < nch * 4) {
+              const uint32_t bd = bd_lo + (uint32_t)(((j >> 2) * Cfg::X_BOX_BYTES + (j & 3) * 32) >> 4);
+              const uint32_t d_t = tmem_base + (j % NACC) * NT;
+              if (j < NACC && seg_first) tc_mma_ts2<false>(d_t, a_t + j * 8, bd, bd_hi, idesc);
+              else tc_mma_ts2<true>(d_t, a_t + j * 8, bd, bd_hi, idesc);
+            }
+          }
+          tc_commit(bar_empty + 8 * cur.stage);
+          tc_commit(bar_aempty + 8 * cur.astage);
+          if (seg_last) tc_commit(bar_accfull);
         }
-        tc_commit(bar_empty + 8 * s);
-        tc_commit(bar_aempty + 8 * t);
-        if (seg_last) {
-          tc_commit(bar_accfull);
-          ++seg;
-        }
-        (void)tile;
+        __syncwarp();
+        if (seg_last) ++seg;
+        cur.template next<STAGES, ASTAGES>(spt);
       }
     }
   } else {
     // ===================== dequant (32 * NDW threads, thread = weight row) + epilogue =====================
     const int row = 32 * (warp & 3) + lane;              // TMEM lane this thread owns
     const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
-    const int sub = (warp - 2) >> 2;                     // which share of a stage's blocks this warp decodes
-    constexpr int SUBS = NDW / 4;
-    const bool epi_warp = (sub == 0);                    // warps 2..5 also run the epilogue
+    const int group = (warp - 2) >> 2;                   // four warps (all TMEM lane quarters) decode one item together
+    constexpr int GROUPS = NDW / 4;
+    static_assert(NDW % 4 == 0 && GROUPS <= ASTAGES, "every dequant group needs an A stage of its own");
+    const bool epi_warp = (group == 0);                  // warps 2..5 also run the epilogue
     const bool leader = (threadIdx.x == 64);
     const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
-    long long n = 0, seg = 0;
-    uint32_t epi_phase = 0;
+    uint32_t seg = 0, epi_phase = 0;
     // all 32 lanes take the same branch after a wait, so the .aligned tcgen05 instructions stay convergent
     auto wait_all = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
       const bool got = mbar_wait(bar, parity, abort_flag);
@@ -394,49 +456,53 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     };
     const uint8_t* ss_bytes = reinterpret_cast<const uint8_t*>(ss_tab);
     const uint8_t* sv_bytes = reinterpret_cast<const uint8_t*>(sv_tab);
-    for (long long it = it_begin; it < it_end; ++it, ++n) {
-      const int s = (int)(n % STAGES), t = (int)(n % ASTAGES);
-      const uint32_t ph = (uint32_t)((n / STAGES) & 1), aph = (uint32_t)((n / ASTAGES) & 1);
-      const long long tile = it / a.steps_per_tile;
-      const int step = (int)(it % a.steps_per_tile);
-      const bool seg_last = (it + 1 == it_end) || step == a.steps_per_tile - 1;
+    const uint32_t mul_lo = a.mul_lo, mul_hi = a.mul_hi;
+    int turn = 0;                                        // item i is decoded by group i % GROUPS
+    for (int i = 0; i < n_items; ++i, cur.template next<STAGES, ASTAGES>(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
+      const int tile = cur.tile, step = cur.step;
+      const bool seg_last = (i + 1 == n_items) || step == spt - 1;
       const int nch = min(CH, a.g.k_chunks - step * CH);
-      if (!wait_all(bar_full + 8 * s, ph, 5)) break;
-      if (!wait_all(bar_aempty + 8 * t, aph ^ 1u, 6)) break;
+      if (turn == group) {
+      if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 5)) break;
+      if (!wait_all(bar_aempty + 8 * cur.astage, (uint32_t)cur.aphase ^ 1u, 6)) break;
       tc_fence_after();
-      const uint8_t* st = smem + (size_t)s * Cfg::STAGE_BYTES;
-      const uint32_t a_t = tmem_a0 + t * Cfg::A_STAGE_COLS + lane_off;
-      for (int c = 0; c < nch; ++c) {
-        const uint8_t* ck = st + c * CHUNK_BYTES;
-        const uint32_t sw = *reinterpret_cast<const uint32_t*>(ck + CHUNK_CODE_BYTES + row * 4);
+      const uint8_t* st = smem + (size_t)cur.stage * Cfg::STAGE_BYTES;
+      const uint32_t a_t = tmem_a0 + cur.astage * Cfg::A_STAGE_COLS + lane_off;
 #pragma unroll
-        for (int bq = 0; bq < CHUNK_BLOCKS / SUBS; ++bq) {
-          const int blk = bq * SUBS + sub;
-          const uint2 cw = *reinterpret_cast<const uint2*>(ck + (blk * TILE_ROWS + row) * 8);
-          // byte offsets into the two tables, straight from the scale word
-          const uint32_t off_ss = (blk == 0 ? sw << 2 : sw >> (8 * blk - 2)) & 0x3FCu;
-          const uint32_t off_sv = (sw >> (8 * blk + 2)) & 0x10u;
-          const uint32_t ss2 = *reinterpret_cast<const uint32_t*>(ss_bytes + off_ss);
-          const SvConsts svc = *reinterpret_cast<const SvConsts*>(sv_bytes + off_sv);
-          uint32_t v[8];
-          decode_word(cw.x, ss2, svc, a.mul_lo, a.mul_hi, v);
-          decode_word(cw.y, ss2, svc, a.mul_lo, a.mul_hi, v + 4);
-          tc_st8(a_t + (c * 4 + blk) * 8, v);
+      for (int c = 0; c < CH; ++c) {
+        if (c < nch) {
+          const uint8_t* ck = st + c * CHUNK_BYTES;
+          const uint32_t sw = *reinterpret_cast<const uint32_t*>(ck + CHUNK_CODE_BYTES + row * 4);
+#pragma unroll
+          for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
+            const uint2 cw = *reinterpret_cast<const uint2*>(ck + (blk * TILE_ROWS + row) * 8);
+            // byte offsets into the two tables, straight from the scale word
+            const uint32_t off_ss = (sw >> (8 * blk) << 2) & 0x3FCu;
+            const uint32_t off_sv = (sw >> (8 * blk + 2)) & 0x10u;
+            const uint32_t ss2 = *reinterpret_cast<const uint32_t*>(ss_bytes + off_ss);
+            const SvConsts svc = *reinterpret_cast<const SvConsts*>(sv_bytes + off_sv);
+            uint32_t v[8];
+            decode_word(cw.x, ss2, svc, mul_lo, mul_hi, v);
+            decode_word(cw.y, ss2, svc, mul_lo, mul_hi, v + 4);
+            tc_st8(a_t + (c * 4 + blk) * 8, v);
+          }
         }
       }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_afull + 8 * t);
+      mbar_arrive(bar_afull + 8 * cur.astage);
+      }
 
       if (!seg_last || !epi_warp) continue;
       // ---------------- epilogue of the segment that ends with this item ----------------
-      const long long tile_begin = tile * a.steps_per_tile;
-      const long long seg_begin = it_begin > tile_begin ? it_begin : tile_begin;
-      const bool complete = (seg_begin == tile_begin) && (step == a.steps_per_tile - 1);
-      const int rt = (int)(tile / a.token_tiles), tt = (int)(tile % a.token_tiles);
+      const int it = it_begin + i;
+      const int tile_begin = tile * spt;
+      const int seg_begin = it_begin > tile_begin ? it_begin : tile_begin;
+      const bool complete = (seg_begin == tile_begin) && (step == spt - 1);
+      const int rt = tile / a.token_tiles, tt = tile - rt * a.token_tiles;
       const int n_out = rt * TILE_ROWS + row;
       const int m0 = tt * NT;
-      if (!wait_all(bar_accfull, (uint32_t)(seg & 1), 7)) break;
+      if (!wait_all(bar_accfull, seg & 1u, 7)) break;
       tc_fence_after();
       const int slot_idx = (seg_begin == it_begin) ? 0 : 1;          // first segment of the stripe or not
       float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(NT * TILE_ROWS);
@@ -445,6 +511,14 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         uint32_t v[16];
         tc_ld16(tmem_base + lane_off + c0, v);
         tc_wait_ld();
+#pragma unroll
+        for (int q = 1; q < NACC; ++q) {
+          uint32_t w[16];
+          tc_ld16(tmem_base + lane_off + q * NT + c0, w);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+        }
         if (complete) {
           if (n_out < a.g.N) {
 #pragma unroll
@@ -465,7 +539,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       // ---------------- partial tile: publish, count, last arrival reduces ----------------
       __threadfence();
       if (!epi_sync()) break;
-      const long long tile_end = tile_begin + a.steps_per_tile;
+      const int tile_end = tile_begin + spt;
       const int c_first = cta_of_item(tile_begin, grid, a.total_items);
       const int c_last = cta_of_item(tile_end - 1, grid, a.total_items);
       if (leader) {
@@ -487,7 +561,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
         for (int c = c_first; c <= c_last; ++c) {
           const long long b_c = (a.total_items * c) / grid;
-          const int sl = (b_c / a.steps_per_tile == tile) ? 0 : 1;
+          const int sl = (b_c / spt == tile) ? 0 : 1;
           const float* src = a.slots + ((size_t)c * 2 + sl) * (size_t)(NT * TILE_ROWS);
 #pragma unroll
           for (int j = 0; j < 16; ++j) acc[j] += __ldcg(src + (c0 + j) * TILE_ROWS + row);
@@ -500,6 +574,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
           }
         }
       }
+      (void)it;
     }
   }
 
@@ -553,7 +628,8 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
+  static const int ch_small = [] { const char* e = getenv("RAZER_CH"); return e ? atoi(e) : 4; }();   // tuning aid: 2, 3 or 4
+  p.CH = p.NT == 16 ? ch_small : p.NT == 32 ? (ch_small == 2 ? 2 : 4) : p.NT == 64 ? 2 : 1;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -585,17 +661,17 @@ size_t umma_workspace_zero_bytes(const razer_desc* d, int M) {
   return WS_STATUS_BYTES + make_plan(d, M).counters_bytes;
 }
 
-template <int NT, int CH, int STAGES, int ASTAGES>
+template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC>
 static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, cudaStream_t st) {
-  using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES>;
-  auto kern = razer_umma_kernel<NT, CH, STAGES, ASTAGES>;
+  using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES, NACC>;
+  auto kern = razer_umma_kernel<NT, CH, STAGES, ASTAGES, NDW, NACC>;
   static bool attr_set = false;
   if (!attr_set) {
     RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES),
                          "cudaFuncSetAttribute(max dynamic shared memory)"));
     attr_set = true;
   }
-  kern<<<grid, UMMA_THREADS, Cfg::SMEM_BYTES, st>>>(tmap, args);
+  kern<<<grid, 64 + 32 * NDW, Cfg::SMEM_BYTES, st>>>(tmap, args);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "razer_umma_kernel launch");
 }
@@ -610,13 +686,27 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   EncodeTiledFn enc = encode_fn();
   if (!enc) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
   CUtensorMap tmap;
-  const cuuint64_t dims[2] = {(cuuint64_t)d->K, (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)ldx_K * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)CHUNK_K, (cuuint32_t)p.NT};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = CUDA_ERROR_UNKNOWN;
+  int map_3d = 0;
+  if (d->K % CHUNK_K == 0 && ldx_K == d->K) {
+    // (64 k, tokens, k chunk) view of x: one box brings the activations of all CH chunks of a stage
+    const cuuint64_t dims[3] = {(cuuint64_t)CHUNK_K, (cuuint64_t)M, (cuuint64_t)(d->K / CHUNK_K)};
+    const cuuint64_t strides[2] = {(cuuint64_t)ldx_K * 2, (cuuint64_t)CHUNK_K * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)CHUNK_K, (cuuint32_t)p.NT, (cuuint32_t)p.CH};
+    r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    map_3d = (r == CUDA_SUCCESS);
+  }
+  if (!map_3d) {
+    const cuuint64_t dims[2] = {(cuuint64_t)d->K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx_K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)CHUNK_K, (cuuint32_t)p.NT};
+    r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   if (r != CUDA_SUCCESS) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
 
   UmmaArgs a;
@@ -636,12 +726,19 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   a.token_tiles = p.token_tiles;
   a.steps_per_tile = p.steps_per_tile;
   a.total_items = p.total_items;
+  a.x_map_3d = map_3d;
+  static const int ndw = [] { const char* e = getenv("RAZER_NDW"); return e ? atoi(e) : 8; }();   // tuning aid
   switch (p.NT) {
-    case 16: return launch_cfg<16, 4, 6, 2>(tmap, a, p.grid, st);
-    case 32: return launch_cfg<32, 4, 5, 2>(tmap, a, p.grid, st);
-    case 64: return launch_cfg<64, 2, 6, 4>(tmap, a, p.grid, st);
-    case 128: return launch_cfg<128, 1, 8, 4>(tmap, a, p.grid, st);
-    default: return launch_cfg<256, 1, 5, 4>(tmap, a, p.grid, st);
+    case 16:
+      if (p.CH == 2) return launch_cfg<16, 2, 10, 6, 16, 4>(tmap, a, p.grid, st);
+      if (p.CH == 3) return launch_cfg<16, 3, 8, 4, 16, 4>(tmap, a, p.grid, st);
+      return ndw == 8 ? launch_cfg<16, 4, 6, 3, 8, 4>(tmap, a, p.grid, st) : launch_cfg<16, 4, 6, 3, 12, 4>(tmap, a, p.grid, st);
+    case 32:
+      if (p.CH == 2) return launch_cfg<32, 2, 10, 6, 16, 2>(tmap, a, p.grid, st);
+      return launch_cfg<32, 4, 5, 3, 12, 2>(tmap, a, p.grid, st);
+    case 64: return launch_cfg<64, 2, 6, 4, 16, 2>(tmap, a, p.grid, st);
+    case 128: return launch_cfg<128, 1, 8, 4, 16, 1>(tmap, a, p.grid, st);
+    default: return launch_cfg<256, 1, 5, 4, 16, 1>(tmap, a, p.grid, st);
   }
 }
 
