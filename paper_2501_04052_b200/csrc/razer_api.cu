@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cmath>
 #include <atomic>
+#include <cstdlib>
 
 #include "razer_common.cuh"
 
@@ -72,6 +73,18 @@ int launch_gemm_umma(const razer_desc*, const void* packed, const void* x, int M
                      const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
 size_t umma_workspace_bytes(const razer_desc*, int M);
 bool umma_supported(const razer_desc*, int M);
+int launch_gemv_mma(const razer_desc*, const void* packed, const void* x, int M, float extra_scale,
+                    const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
+size_t gemv_mma_workspace_bytes(const razer_desc*, int M);
+bool gemv_mma_supported(const razer_desc*, int M);
+
+// Kernel choice: register-fragment MMA kernel for M <= 16, tcgen05 kernel above.
+// RAZER_KERNEL=simt / umma (environment, debugging aid) force the CUDA-core / tcgen05 kernel.
+static char kernel_override() {
+  static const char c = [] { const char* e = getenv("RAZER_KERNEL"); return e ? e[0] : '\0'; }();
+  return c;
+}
+static bool use_mma(const razer_desc* d, int M) { return kernel_override() == '\0' && gemv_mma_supported(d, M); }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -122,10 +135,12 @@ int razer_workspace_bytes(const razer_desc* d, int M, int op, size_t* bytes_out)
     case RAZER_OP_GEMM:
       b = simt_workspace_bytes(d, M);
       if (umma_supported(d, M)) b = b > umma_workspace_bytes(d, M) ? b : umma_workspace_bytes(d, M);
+      if (gemv_mma_supported(d, M)) b = b > gemv_mma_workspace_bytes(d, M) ? b : gemv_mma_workspace_bytes(d, M);
       break;
     case RAZER_OP_GEMM_W4A4: {
       size_t g = simt_workspace_bytes(d, M);
       if (umma_supported(d, M)) g = g > umma_workspace_bytes(d, M) ? g : umma_workspace_bytes(d, M);
+      if (gemv_mma_supported(d, M)) g = g > gemv_mma_workspace_bytes(d, M) ? g : gemv_mma_workspace_bytes(d, M);
       b = align_up((size_t)M * d->K * 2, 256) + g;
       break;
     }
@@ -160,6 +175,8 @@ static int matmul_common(const razer_desc* d, const void* packed_dev, const void
   RAZER_TRY(check_ptr(y_dev, 2, "y_dev"));
   if (ws && reinterpret_cast<uintptr_t>(ws) % 256)
     return set_error(RAZER_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+  if (use_mma(d, M))
+    return launch_gemv_mma(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   if (umma_supported(d, M))
     return launch_gemm_umma(d, packed_dev, x_dev, M, d->K, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   razer_desc dd = *d;

@@ -16,7 +16,11 @@ namespace razer {
 //
 // The tensor is cut into tiles of TILE_ROWS rows x CHUNK_K columns (4 blocks of 16).
 // One tile-chunk is CHUNK_BYTES contiguous bytes:
-//   [blk 0..3][row 0..127] 8 bytes : the block's 16 nibbles as two 32-bit words; element j of
+//   [blk 0..3][slot 0..127] 8 bytes: the block's 16 nibbles as two 32-bit words; row r sits in
+//                                    slot r for even blocks and r ^ 8 for odd ones (so that a
+//                                    warp reading rows g, g+1.. of four different blocks, the
+//                                    tensor-core fragment pattern, meets no bank conflict, while
+//                                    thread = row reads stay contiguous); element j of
 //                                    the block sits in word j/8, nibble (j%8)/2 + 4*(j%2), so
 //                                    that nibbles p and p+4 of a word (the same position in
 //                                    its two 16-bit halves) are elements 2p and 2p+1
@@ -30,7 +34,7 @@ namespace razer {
 //     nibble is S E1 E0 M as in Eq. 5;
 //   * a block whose special value is negative is stored negated (sign bits of all non-zero
 //     codes flipped) so that nibble 0x0 always means "+sv_mag[select]";
-//   * scale byte = [negate | select | 6-bit scale code]; negate = 1 means the block's
+//   * scale byte = [select | negate | 6-bit scale code]; negate = 1 means the block's
 //     values are the negatives of the stored codes' values.
 // With these conventions the decoder needs no comparison: the nibble's bits drop into a
 // bf16 bit pattern (sign to bit 15, E1 E0 M to bits 8:6, value x 2^-126), the special value
@@ -103,6 +107,13 @@ __device__ __forceinline__ float scale_value(uint32_t code) {
   const float normal = __uint_as_float(((120u + e) << 23) | (m << 20));
   return e ? normal : (float)m * 0.001953125f;   // m * 2^-9
 }
+
+// Slot of row `row_in` (0..127) in block `blk` of a chunk, and the byte offset of its code words.
+__host__ __device__ __forceinline__ int packed_slot(int blk, int row_in) { return row_in ^ ((blk & 1) << 3); }
+__host__ __device__ __forceinline__ int packed_code_offset(int blk, int row_in) {
+  return (blk * TILE_ROWS + packed_slot(blk, row_in)) * 8;
+}
+constexpr uint32_t PACKED_NEGATE = 0x40u, PACKED_SELECT = 0x80u;   // bits of a packed scale byte
 
 // Position (in bits) of element j's nibble inside the block's 64-bit code word.
 __host__ __device__ __forceinline__ int packed_nibble_shift(int j) {

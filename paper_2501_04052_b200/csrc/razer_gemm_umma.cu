@@ -15,12 +15,7 @@
 // warps w and w + 4 own the same 32 weight rows and split the stage's blocks between them;
 // the first four dequant warps also run the epilogue of the tile they just fed.
 //
-// Decode (per pair of elements, no comparison, no conversion instruction): the stored nibble
-// is isolated in both 16-bit halves of the word, one integer multiply-add drops two shifted
-// copies of it, one logic op keeps sign -> bit 15 and E1 E0 M -> bits 8:6 (a bf16 pattern worth
-// value x 2^-126, subnormal for 0.5) and ORs in the special value, which one fused
-// multiply-add with ReLU derives from the isolated nibble (it is the only nibble that is
-// numerically zero); one packed bf16 multiply by +-scale x 2^126 finishes the exact product.
+// The register-level decode is described in razer_decode.cuh.
 //
 // Work partition (Sec. 4.3 / App. E of the paper: stripes of about equal length that may span
 // several output tiles, partial results reduced through global memory): the grid is
@@ -36,6 +31,7 @@
 #include <cstdlib>
 
 #include "razer_common.cuh"
+#include "razer_decode.cuh"
 
 namespace razer {
 
@@ -174,50 +170,6 @@ __host__ __device__ constexpr uint32_t make_idesc(int nt) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// ------------------------------------------------------------------ decode (registers)
-__device__ __forceinline__ uint32_t fma_relu_bf16x2(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("fma.rn.relu.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
-  uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-
-// Per-block decode constants, looked up in shared memory by the block's scale byte.
-struct SvConsts {            // indexed by the select bit
-  uint32_t sv;               // (sv, sv) x 2^-126 as bf16x2
-  uint32_t nsv_lo;           // -(sv x 2^7):  sv_pattern - nsv_lo * (nibble in bits 3:0 read as bf16) = 0 for nibble 1
-  uint32_t nsv_hi;           // -(sv x 2^3):  the same for a nibble in bits 7:4
-  uint32_t pad;
-};
-
-// Four stored nibbles of each 16-bit half of `w` -> four bf16x2 registers (elements 2p, 2p+1
-// of the word in register p), each the exact product value x scale with the block's sign.
-__device__ __forceinline__ void decode_word(uint32_t w, uint32_t ss2, const SvConsts& c, uint32_t mul_lo,
-                                            uint32_t mul_hi, uint32_t* out) {
-  const uint32_t w8 = w >> 8;
-  const uint32_t n0 = w & 0x000F000Fu, n1 = w & 0x00F000F0u;
-  const uint32_t n2 = w8 & 0x000F000Fu, n3 = w8 & 0x00F000F0u;
-  // nibble * (2^6 + 2^12) [bits 3:0] or * (2^2 + 2^8) [bits 7:4]: one copy lands with E1 E0 M on
-  // bits 8:6, the other with S on bit 15; the mask keeps exactly those
-  const uint32_t u0 = and_or(n0 * mul_lo, 0x81C081C0u, fma_relu_bf16x2(n0, c.nsv_lo, c.sv));
-  const uint32_t u1 = and_or(n1 * mul_hi, 0x81C081C0u, fma_relu_bf16x2(n1, c.nsv_hi, c.sv));
-  const uint32_t u2 = and_or(n2 * mul_lo, 0x81C081C0u, fma_relu_bf16x2(n2, c.nsv_lo, c.sv));
-  const uint32_t u3 = and_or(n3 * mul_hi, 0x81C081C0u, fma_relu_bf16x2(n3, c.nsv_hi, c.sv));
-  out[0] = mul_bf16x2(u0, ss2);
-  out[1] = mul_bf16x2(u1, ss2);
-  out[2] = mul_bf16x2(u2, ss2);
-  out[3] = mul_bf16x2(u3, ss2);
-}
-
 // ------------------------------------------------------------------ kernel
 struct UmmaArgs {
   const uint8_t* packed;
@@ -247,7 +199,7 @@ struct UmmaCfg {
   static constexpr int TMEM_COLS = TMEM_COLS_NEEDED <= 64 ? 64 : TMEM_COLS_NEEDED <= 128 ? 128
                                    : TMEM_COLS_NEEDED <= 256 ? 256 : 512;
   static constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 3;
-  static constexpr int TABLE_BYTES = 256 * 4 + 2 * 16;         // scale-byte table + special-value constants
+  static constexpr int TABLE_BYTES = DECODE_TABLE_BYTES;        // scale table + special-value constants
   static constexpr size_t SMEM_BYTES =
       1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + NUM_BARS * 8 + 16 + 64 + TABLE_BYTES;
   static_assert(TMEM_COLS_NEEDED <= 512, "TMEM budget exceeded");
@@ -284,8 +236,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       (reinterpret_cast<uintptr_t>(bars + Cfg::NUM_BARS) + 15) & ~(uintptr_t)15);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   uint32_t* bcast = tmem_slot + 2;                      // epilogue broadcast word
-  uint32_t* ss_tab = tmem_slot + 16;                    // [256] (+-scale x 2^126) as bf16x2, by scale byte
-  SvConsts* sv_tab = reinterpret_cast<SvConsts*>(ss_tab + 256);   // [2] by select bit
+  uint8_t* tables = reinterpret_cast<uint8_t*>(tmem_slot + 16);   // decode tables (razer_decode.cuh)
 
   const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> dequant, MMA
   const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]  MMA commit -> TMA
@@ -322,24 +273,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = threadIdx.x; i < 256; i += THREADS) {
-    // scale x 2^126 has four significant bits: the upper half of the FP32 pattern is the exact bf16
-    const float sc = scale_value((uint32_t)i & 0x3Fu) * 8.50705917e37f;   // 2^126
-    const uint32_t b = (__float_as_uint(sc) >> 16) | (((uint32_t)i & 0x80u) << 8);
-    ss_tab[i] = b | (b << 16);
-  }
-  if (threadIdx.x < 2) {
-    const float sv = threadIdx.x ? a.sv1 : a.sv0;          // at most four significant bits
-    const uint32_t p0 = __float_as_uint(sv * 1.17549435e-38f) >> 16;     // sv x 2^-126
-    const uint32_t p1 = __float_as_uint(-sv * 128.0f) >> 16;
-    const uint32_t p2 = __float_as_uint(-sv * 8.0f) >> 16;
-    SvConsts c;
-    c.sv = p0 | (p0 << 16);
-    c.nsv_lo = p1 | (p1 << 16);
-    c.nsv_hi = p2 | (p2 << 16);
-    c.pad = 0;
-    sv_tab[threadIdx.x] = c;
-  }
+  decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x, THREADS);
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"((uint32_t)Cfg::TMEM_COLS)
@@ -454,8 +388,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       ++epi_phase;
       return got;
     };
-    const uint8_t* ss_bytes = reinterpret_cast<const uint8_t*>(ss_tab);
-    const uint8_t* sv_bytes = reinterpret_cast<const uint8_t*>(sv_tab);
+    const DecodeTables dt = decode_tables_view(tables, lane);
     const uint32_t mul_lo = a.mul_lo, mul_hi = a.mul_hi;
     int turn = 0;                                        // item i is decoded by group i % GROUPS
     for (int i = 0; i < n_items; ++i, cur.template next<STAGES, ASTAGES>(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
@@ -475,12 +408,10 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
           const uint32_t sw = *reinterpret_cast<const uint32_t*>(ck + CHUNK_CODE_BYTES + row * 4);
 #pragma unroll
           for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
-            const uint2 cw = *reinterpret_cast<const uint2*>(ck + (blk * TILE_ROWS + row) * 8);
-            // byte offsets into the two tables, straight from the scale word
-            const uint32_t off_ss = (sw >> (8 * blk) << 2) & 0x3FCu;
-            const uint32_t off_sv = (sw >> (8 * blk + 2)) & 0x10u;
-            const uint32_t ss2 = *reinterpret_cast<const uint32_t*>(ss_bytes + off_ss);
-            const SvConsts svc = *reinterpret_cast<const SvConsts*>(sv_bytes + off_sv);
+            const uint2 cw = *reinterpret_cast<const uint2*>(ck + packed_code_offset(blk, row));
+            uint32_t ss2;
+            SvConsts svc;
+            decode_block_consts(dt, sw, blk, ss2, svc);
             uint32_t v[8];
             decode_word(cw.x, ss2, svc, mul_lo, mul_hi, v);
             decode_word(cw.y, ss2, svc, mul_lo, mul_hi, v + 4);

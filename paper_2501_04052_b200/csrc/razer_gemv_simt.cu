@@ -42,11 +42,11 @@ gemv_simt_kernel(const uint8_t* __restrict__ packed, const __nv_bfloat16* __rest
       const uint32_t sw = *reinterpret_cast<const uint32_t*>(base + CHUNK_CODE_BYTES + row_in * 4);
 #pragma unroll
       for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
-        const uint2 cw = *reinterpret_cast<const uint2*>(base + ((size_t)blk * TILE_ROWS + row_in) * 8);
+        const uint2 cw = *reinterpret_cast<const uint2*>(base + packed_code_offset(blk, row_in));
         const uint32_t sb = (sw >> (8 * blk)) & 0xFFu;
         float s = scale_value(sb & 0x3Fu);
-        if (sb & 0x80u) s = -s;
-        const float sv = (sb & 0x40u) ? sv1 : sv0;
+        if (sb & PACKED_NEGATE) s = -s;
+        const float sv = (sb & PACKED_SELECT) ? sv1 : sv0;
         float part[MT];
 #pragma unroll
         for (int m = 0; m < MT; ++m) part[m] = 0.0f;

@@ -43,14 +43,14 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __
     const bool negate = (sb & 0x80u) != 0;              // negative special value: store the block negated
     uint32_t out_sb = 0;
     if (scode != 0) {
-      out_sb = (negate ? 0x80u : 0u) | (sb & 0x40u) | scode;
+      out_sb = (negate ? PACKED_NEGATE : 0u) | ((sb & 0x40u) ? PACKED_SELECT : 0u) | scode;
       w0 = shuffle(canon(w0, negate));
       w1 = shuffle(canon(w1, negate));
     } else {
       w0 = w1 = 0x88888888u;                            // zero block: sixteen true zeros
     }
     uint8_t* base = packed + (size_t)chunk * CHUNK_BYTES;
-    *reinterpret_cast<uint2*>(base + ((size_t)blk * TILE_ROWS + row_in) * 8) = make_uint2(w0, w1);
+    *reinterpret_cast<uint2*>(base + packed_code_offset(blk, row_in)) = make_uint2(w0, w1);
     base[CHUNK_CODE_BYTES + row_in * 4 + blk] = (uint8_t)out_sb;
   }
 }
@@ -72,11 +72,11 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ packed, void* __restr
     const int k0 = (kc * CHUNK_BLOCKS + blk) * 16;
     if (n >= g.N || k0 >= g.K) continue;
     const uint8_t* base = packed + (size_t)chunk * CHUNK_BYTES;
-    const uint2 c = *reinterpret_cast<const uint2*>(base + ((size_t)blk * TILE_ROWS + row_in) * 8);
+    const uint2 c = *reinterpret_cast<const uint2*>(base + packed_code_offset(blk, row_in));
     const uint32_t sb = base[CHUNK_CODE_BYTES + row_in * 4 + blk];
     float s = scale_value(sb & 0x3Fu);
-    if (sb & 0x80u) s = -s;
-    const float sv = p.sv_mag[(sb >> 6) & 1u];
+    if (sb & PACKED_NEGATE) s = -s;
+    const float sv = p.sv_mag[(sb & PACKED_SELECT) ? 1 : 0];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
       float d1 = packed_elem(packed_nibble(c, j), sv) * s;   // exact: <= 8 significant bits
