@@ -224,7 +224,10 @@ struct ItemCursor {
   }
 };
 
-template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC>
+// GI ("group issue"): each dequant group issues the MMAs of the items it decoded itself, into accumulators
+// of its own, instead of handing them to the MMA warp.  Used for narrow token tiles, where an item's MMAs
+// are short and one issuing warp per CTA would be the serial bottleneck.
+template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC, bool GI>
 __global__ void __launch_bounds__(64 + 32 * NDW, 1)
 razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) {
   using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES, NACC>;
@@ -266,7 +269,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       mbar_init(bar_afull + 8 * i, 128);
       mbar_init(bar_aempty + 8 * i, 1);
     }
-    mbar_init(bar_accfull, 1);
+    mbar_init(bar_accfull, GI ? NDW / 4 : 1);
     mbar_init(bar_accempty, 128);
     mbar_init(bar_epi, 128);
     *abort_flag = 0;
@@ -322,7 +325,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     }
   } else if (warp == 1) {
     // ===================== MMA issuer (whole warp walks the items, one elected lane issues) =====================
-    {
+    if (!GI) {
       constexpr uint32_t idesc = make_idesc(NT);
       // upper half of the shared-memory descriptor: 1024-byte group stride, descriptor version, 128-byte swizzle
       constexpr uint32_t bd_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -372,6 +375,11 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     const int group = (warp - 2) >> 2;                   // four warps (all TMEM lane quarters) decode one item together
     constexpr int GROUPS = NDW / 4;
     static_assert(NDW % 4 == 0 && GROUPS <= ASTAGES, "every dequant group needs an A stage of its own");
+    static_assert(!GI || (NACC % GROUPS == 0 && ASTAGES == GROUPS), "group issue: A stage and accumulators per group");
+    constexpr int APG = GI ? NACC / GROUPS : NACC;       // accumulators per group
+    const bool issuer = GI && ((warp - 2) & 3) == 0;     // first warp of a group issues the group's MMAs
+    uint32_t own_phase = 0, gseg = 0;                    // GI: parity of the group's A stage; segments seen
+    bool fresh = true;                                   // GI: the group's accumulators hold nothing of this segment yet
     const bool epi_warp = (group == 0);                  // warps 2..5 also run the epilogue
     const bool leader = (threadIdx.x == 64);
     const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
@@ -395,12 +403,20 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       const int tile = cur.tile, step = cur.step;
       const bool seg_last = (i + 1 == n_items) || step == spt - 1;
       const int nch = min(CH, a.g.k_chunks - step * CH);
+      const bool seg_first = (i == 0) || step == 0;
+      if (GI && seg_first) {
+        fresh = true;
+        // the epilogue of the previous segment must have read the accumulators before any group moves on
+        if (issuer && gseg > 0 && !wait_all(bar_accempty, (gseg & 1u) ^ 1u, 4)) break;
+      }
       if (turn == group) {
+      const int astage = GI ? group : cur.astage;
+      const uint32_t aph = GI ? own_phase : (uint32_t)cur.aphase;
       if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 5)) break;
-      if (!wait_all(bar_aempty + 8 * cur.astage, (uint32_t)cur.aphase ^ 1u, 6)) break;
+      if (!wait_all(bar_aempty + 8 * astage, aph ^ 1u, 6)) break;
       tc_fence_after();
       const uint8_t* st = smem + (size_t)cur.stage * Cfg::STAGE_BYTES;
-      const uint32_t a_t = tmem_a0 + cur.astage * Cfg::A_STAGE_COLS + lane_off;
+      const uint32_t a_t = tmem_a0 + astage * Cfg::A_STAGE_COLS + lane_off;
 #pragma unroll
       for (int c = 0; c < CH; ++c) {
         if (c < nch) {
@@ -421,7 +437,43 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_afull + 8 * cur.astage);
+      mbar_arrive(bar_afull + 8 * astage);
+      if (GI) {
+        if (issuer) {
+          // the group's 128 threads have stored their rows: issue this item's MMAs from here
+          if (!wait_all(bar_afull + 8 * astage, aph, 3)) break;
+          tc_fence_after();
+          constexpr uint32_t idesc = make_idesc(NT);
+          constexpr uint32_t bd_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+          const uint32_t xs = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES + Cfg::W_PAD;
+          const uint32_t bd_lo = (xs >> 4) | (1u << 16);
+          const uint32_t a_s = tmem_a0 + astage * Cfg::A_STAGE_COLS;
+          if (elect_one()) {
+#pragma unroll
+            for (int j = 0; j < CH * 4; ++j) {
+              if (j < nch * 4) {
+                const uint32_t bd = bd_lo + (uint32_t)(((j >> 2) * Cfg::X_BOX_BYTES + (j & 3) * 32) >> 4);
+                const uint32_t d_t = tmem_base + (group * APG + j % APG) * NT;
+                if (j < APG && fresh) tc_mma_ts2<false>(d_t, a_s + j * 8, bd, bd_hi, idesc);
+                else tc_mma_ts2<true>(d_t, a_s + j * 8, bd, bd_hi, idesc);
+              }
+            }
+            tc_commit(bar_empty + 8 * cur.stage);
+            tc_commit(bar_aempty + 8 * astage);
+          }
+          __syncwarp();
+        }
+        fresh = false;
+        own_phase ^= 1u;
+      }
+      }
+      if (GI && seg_last) {
+        // every group reports its share of the segment (a group without an item in it reports at once)
+        if (issuer) {
+          if (elect_one()) tc_commit(bar_accfull);
+          __syncwarp();
+        }
+        ++gseg;
       }
 
       if (!seg_last || !epi_warp) continue;
@@ -437,18 +489,30 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       tc_fence_after();
       const int slot_idx = (seg_begin == it_begin) ? 0 : 1;          // first segment of the stripe or not
       float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(NT * TILE_ROWS);
+      bool acc_valid[GROUPS];                                         // GI: which groups had an item in this segment
+      {
+        const int i0 = seg_begin - it_begin, len = i - i0 + 1;
+#pragma unroll
+        for (int q = 0; q < GROUPS; ++q) acc_valid[q] = (len >= GROUPS) || (((q - i0 % GROUPS + GROUPS) % GROUPS) < len);
+      }
 #pragma unroll 1
       for (int c0 = 0; c0 < NT; c0 += 16) {
         uint32_t v[16];
         tc_ld16(tmem_base + lane_off + c0, v);
         tc_wait_ld();
+        if (GI && !acc_valid[0]) {                                    // group 0 had no item in this segment
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0;
+        }
 #pragma unroll
         for (int q = 1; q < NACC; ++q) {
           uint32_t w[16];
           tc_ld16(tmem_base + lane_off + q * NT + c0, w);
           tc_wait_ld();
+          if (!GI || acc_valid[q / APG]) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+            for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+          }
         }
         if (complete) {
           if (n_out < a.g.N) {
@@ -559,8 +623,7 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  static const int ch_small = [] { const char* e = getenv("RAZER_CH"); return e ? atoi(e) : 4; }();   // tuning aid: 2, 3 or 4
-  p.CH = p.NT == 16 ? ch_small : p.NT == 32 ? (ch_small == 2 ? 2 : 4) : p.NT == 64 ? 2 : 1;
+  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -592,10 +655,10 @@ size_t umma_workspace_zero_bytes(const razer_desc* d, int M) {
   return WS_STATUS_BYTES + make_plan(d, M).counters_bytes;
 }
 
-template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC>
+template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC, bool GI>
 static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, cudaStream_t st) {
   using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES, NACC>;
-  auto kern = razer_umma_kernel<NT, CH, STAGES, ASTAGES, NDW, NACC>;
+  auto kern = razer_umma_kernel<NT, CH, STAGES, ASTAGES, NDW, NACC, GI>;
   static bool attr_set = false;
   if (!attr_set) {
     RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES),
@@ -661,15 +724,12 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   static const int ndw = [] { const char* e = getenv("RAZER_NDW"); return e ? atoi(e) : 8; }();   // tuning aid
   switch (p.NT) {
     case 16:
-      if (p.CH == 2) return launch_cfg<16, 2, 10, 6, 16, 4>(tmap, a, p.grid, st);
-      if (p.CH == 3) return launch_cfg<16, 3, 8, 4, 16, 4>(tmap, a, p.grid, st);
-      return ndw == 8 ? launch_cfg<16, 4, 6, 3, 8, 4>(tmap, a, p.grid, st) : launch_cfg<16, 4, 6, 3, 12, 4>(tmap, a, p.grid, st);
-    case 32:
-      if (p.CH == 2) return launch_cfg<32, 2, 10, 6, 16, 2>(tmap, a, p.grid, st);
-      return launch_cfg<32, 4, 5, 3, 12, 2>(tmap, a, p.grid, st);
-    case 64: return launch_cfg<64, 2, 6, 4, 16, 2>(tmap, a, p.grid, st);
-    case 128: return launch_cfg<128, 1, 8, 4, 16, 1>(tmap, a, p.grid, st);
-    default: return launch_cfg<256, 1, 5, 4, 16, 1>(tmap, a, p.grid, st);
+      if (ndw == 8) return launch_cfg<16, 4, 6, 3, 12, 4, false>(tmap, a, p.grid, st);   // tuning aid: MMA-warp issue
+      return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
+    case 32: return launch_cfg<32, 4, 5, 3, 12, 3, true>(tmap, a, p.grid, st);
+    case 64: return launch_cfg<64, 2, 6, 4, 16, 4, true>(tmap, a, p.grid, st);
+    case 128: return launch_cfg<128, 1, 8, 4, 16, 1, false>(tmap, a, p.grid, st);
+    default: return launch_cfg<256, 1, 5, 4, 16, 1, false>(tmap, a, p.grid, st);
   }
 }
 
