@@ -78,13 +78,14 @@ int launch_gemv_mma(const razer_desc*, const void* packed, const void* x, int M,
 size_t gemv_mma_workspace_bytes(const razer_desc*, int M);
 bool gemv_mma_supported(const razer_desc*, int M);
 
-// Kernel choice: register-fragment MMA kernel for M <= 16, tcgen05 kernel above.
-// RAZER_KERNEL=simt / umma (environment, debugging aid) force the CUDA-core / tcgen05 kernel.
+// Kernel choice: the tcgen05 kernel serves every M.  RAZER_KERNEL=mma (environment) routes M <= 16 to the
+// register-fragment mma.sync kernel instead (kept for comparison: it measures slower on B200), =simt routes
+// everything to the CUDA-core kernel (debugging aid).
 static char kernel_override() {
   static const char c = [] { const char* e = getenv("RAZER_KERNEL"); return e ? e[0] : '\0'; }();
   return c;
 }
-static bool use_mma(const razer_desc* d, int M) { return kernel_override() == '\0' && gemv_mma_supported(d, M); }
+static bool use_mma(const razer_desc* d, int M) { return kernel_override() == 'm' && gemv_mma_supported(d, M); }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

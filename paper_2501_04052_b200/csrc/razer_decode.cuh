@@ -44,9 +44,9 @@ struct SvConsts {
 constexpr int DECODE_SS_ENTRIES = 128;
 constexpr int DECODE_TABLE_BYTES = DECODE_SS_ENTRIES * 32 * 4 + 2 * 16;
 
-struct DecodeTables {
-  const uint8_t* ss_lane;    // &ss[0][lane]
-  const uint8_t* sv;
+struct DecodeTables {         // 32-bit shared-window addresses
+  uint32_t ss_lane;          // &ss[0][lane]
+  uint32_t sv;
 };
 
 // Fill the tables (all threads of the CTA call this; a __syncthreads() must follow).
@@ -75,8 +75,8 @@ __device__ __forceinline__ void decode_tables_fill(uint8_t* base, float sv0, flo
 
 __device__ __forceinline__ DecodeTables decode_tables_view(const uint8_t* base, int lane) {
   DecodeTables t;
-  t.ss_lane = base + lane * 4;
-  t.sv = base + DECODE_SS_ENTRIES * 32 * 4;
+  t.ss_lane = smem_addr(base) + lane * 4;
+  t.sv = smem_addr(base) + DECODE_SS_ENTRIES * 32 * 4;
   return t;
 }
 
@@ -86,8 +86,22 @@ __device__ __forceinline__ void decode_block_consts(const DecodeTables& t, uint3
                                                     SvConsts& svc) {
   const uint32_t off_ss = (blk == 0 ? sw << 7 : sw >> (8 * blk - 7)) & 0x3F80u;   // (byte & 0x7F) * 128
   const uint32_t off_sv = (sw >> (8 * blk + 3)) & 0x10u;                          // (byte >> 7) * 16
-  ss2 = *reinterpret_cast<const uint32_t*>(t.ss_lane + off_ss);
-  svc = *reinterpret_cast<const SvConsts*>(t.sv + off_sv);
+  ss2 = lds32(t.ss_lane + off_ss);
+  const uint4 c = lds128(t.sv + off_sv);
+  svc.sv = c.x;
+  svc.nsv_lo = c.y;
+  svc.nsv_hi = c.z;
+  svc.pad = 0;
+}
+
+// The same for a scale byte already shifted down to bits 7:0 (higher bits may hold anything).
+__device__ __forceinline__ void decode_block_consts_byte(const DecodeTables& t, uint32_t sb, uint32_t& ss2, SvConsts& svc) {
+  ss2 = lds32(t.ss_lane + ((sb << 7) & 0x3F80u));
+  const uint4 c = lds128(t.sv + ((sb >> 3) & 0x10u));
+  svc.sv = c.x;
+  svc.nsv_lo = c.y;
+  svc.nsv_hi = c.z;
+  svc.pad = 0;
 }
 
 // Four stored nibbles of each 16-bit half of `w` -> four bf16x2 registers (elements 2p, 2p+1

@@ -55,32 +55,35 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One poll of a barrier phase.  The hint lets the hardware park the thread until the phase
+// completes (or about the hinted time passes) instead of spinning in the issue slots that
+// the decoding warps need.
+constexpr uint32_t WAIT_SLICE_NS = 1000000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(WAIT_SLICE_NS)
       : "memory");
   return ok != 0;
 }
-// Bounded wait; false = gave up (or another thread already flagged a failure).
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+// Bounded wait; false = gave up (or another thread already flagged a failure).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  for (uint32_t i = 1; i < WAIT_LIMIT; ++i) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();                     // only waits that already lasted a slice get here
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
-    }
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
   }
   return false;
 }
@@ -415,22 +418,26 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 5)) break;
       if (!wait_all(bar_aempty + 8 * astage, aph ^ 1u, 6)) break;
       tc_fence_after();
-      const uint8_t* st = smem + (size_t)cur.stage * Cfg::STAGE_BYTES;
+      const uint32_t st = smem_addr(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
       const uint32_t a_t = tmem_a0 + astage * Cfg::A_STAGE_COLS + lane_off;
 #pragma unroll
       for (int c = 0; c < CH; ++c) {
         if (c < nch) {
-          const uint8_t* ck = st + c * CHUNK_BYTES;
-          const uint32_t sw = *reinterpret_cast<const uint32_t*>(ck + CHUNK_CODE_BYTES + row * 4);
+          const uint32_t ck = st + c * CHUNK_BYTES;
+          // all of the chunk's loads first, then the arithmetic
+          const uint32_t sw = lds32(ck + CHUNK_CODE_BYTES + row * 4);
+          uint2 cw[CHUNK_BLOCKS];
+#pragma unroll
+          for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) cw[blk] = lds64(ck + packed_code_offset(blk, row));
+          uint32_t ss2[CHUNK_BLOCKS];
+          SvConsts svc[CHUNK_BLOCKS];
+#pragma unroll
+          for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) decode_block_consts(dt, sw, blk, ss2[blk], svc[blk]);
 #pragma unroll
           for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
-            const uint2 cw = *reinterpret_cast<const uint2*>(ck + packed_code_offset(blk, row));
-            uint32_t ss2;
-            SvConsts svc;
-            decode_block_consts(dt, sw, blk, ss2, svc);
             uint32_t v[8];
-            decode_word(cw.x, ss2, svc, mul_lo, mul_hi, v);
-            decode_word(cw.y, ss2, svc, mul_lo, mul_hi, v + 4);
+            decode_word(cw[blk].x, ss2[blk], svc[blk], mul_lo, mul_hi, v);
+            decode_word(cw[blk].y, ss2[blk], svc[blk], mul_lo, mul_hi, v + 4);
             tc_st8(a_t + (c * 4 + blk) * 8, v);
           }
         }
@@ -623,7 +630,8 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
+  static const int ch16 = [] { const char* e = getenv("RAZER_CH"); return e ? atoi(e) : 4; }();   // tuning aid: 3 or 4
+  p.CH = p.NT == 16 ? (ch16 == 3 ? 3 : 4) : p.NT == 32 ? 4 : p.NT == 64 ? 2 : 1;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -721,10 +729,9 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   a.steps_per_tile = p.steps_per_tile;
   a.total_items = p.total_items;
   a.x_map_3d = map_3d;
-  static const int ndw = [] { const char* e = getenv("RAZER_NDW"); return e ? atoi(e) : 8; }();   // tuning aid
   switch (p.NT) {
     case 16:
-      if (ndw == 8) return launch_cfg<16, 4, 6, 3, 12, 4, false>(tmap, a, p.grid, st);   // tuning aid: MMA-warp issue
+      if (p.CH == 3) return launch_cfg<16, 3, 8, 4, 16, 4, true>(tmap, a, p.grid, st);
       return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
     case 32: return launch_cfg<32, 4, 5, 3, 12, 3, true>(tmap, a, p.grid, st);
     case 64: return launch_cfg<64, 2, 6, 4, 16, 4, true>(tmap, a, p.grid, st);

@@ -49,14 +49,18 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One poll of a barrier phase.  The hint lets the hardware park the thread until the phase
+// completes (or about the hinted time passes) instead of spinning in the issue slots that
+// the decoding warps need.
+constexpr uint32_t WAIT_SLICE_NS = 1000000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(WAIT_SLICE_NS)
       : "memory");
   return ok != 0;
 }
@@ -68,13 +72,12 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait; false = gave up (or another thread already flagged a failure).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  for (uint32_t i = 1; i < WAIT_LIMIT; ++i) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();                     // only waits that already lasted a slice get here
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
-    }
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
   }
   return false;
 }
@@ -268,27 +271,28 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
       const bool seg_last = (i + 1 == n_items) || step == spt - 1;
       const int nch = min(CH, a.g.k_chunks - step * CH);
       if (!wait_all(bar_full + 8 * stage, (uint32_t)phase, 24)) break;
-      const uint8_t* st = smem + (size_t)stage * C::STAGE_BYTES;
+      const uint32_t st = smem_addr(smem) + (uint32_t)stage * C::STAGE_BYTES;
 #pragma unroll
       for (int cc = 0; cc < (CH + 1) / 2; ++cc) {
         const int c = 2 * cc + half;
         if (c < nch) {
-          const uint8_t* ck = st + c * CHUNK_BYTES;
-          const uint8_t* xk = st + C::W_PAD + c * C::X_BOX_BYTES;
+          const uint32_t ck = st + c * CHUNK_BYTES;
+          const uint32_t xk = st + C::W_PAD + c * C::X_BOX_BYTES;
           uint2 xb[NTILES][4];
 #pragma unroll
           for (int nt = 0; nt < NTILES; ++nt)
 #pragma unroll
-            for (int q = 0; q < 4; ++q) xb[nt][q] = *reinterpret_cast<const uint2*>(xk + xb_off[nt][q]);
+            for (int q = 0; q < 4; ++q) xb[nt][q] = lds64(xk + xb_off[nt][q]);
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
             uint32_t e[2][8];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-              const uint2 cwd = *reinterpret_cast<const uint2*>(ck + code_off[mt][h]);
-              const uint32_t sb = *reinterpret_cast<const uint32_t*>(ck + scale_off[mt][h]) >> (8 * t);
-              const uint32_t ss2 = *reinterpret_cast<const uint32_t*>(dt.ss_lane + ((sb << 7) & 0x3F80u));
-              const SvConsts svc = *reinterpret_cast<const SvConsts*>(dt.sv + ((sb >> 3) & 0x10u));
+              const uint2 cwd = lds64(ck + code_off[mt][h]);
+              const uint32_t sb = lds32(ck + scale_off[mt][h]) >> (8 * t);
+              uint32_t ss2;
+              SvConsts svc;
+              decode_block_consts_byte(dt, sb, ss2, svc);
               decode_word(cwd.x, ss2, svc, mul_lo, mul_hi, e[h]);
               decode_word(cwd.y, ss2, svc, mul_lo, mul_hi, e[h] + 4);
             }
