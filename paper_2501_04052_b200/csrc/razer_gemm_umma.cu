@@ -273,8 +273,8 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       mbar_init(bar_aempty + 8 * i, 1);
     }
     mbar_init(bar_accfull, GI ? NDW / 4 : 1);
-    mbar_init(bar_accempty, 128);
-    mbar_init(bar_epi, 128);
+    mbar_init(bar_accempty, GI ? 128 : 32 * NDW);         // threads that read the accumulator in the epilogue
+    mbar_init(bar_epi, GI ? 128 : 32 * NDW);
     *abort_flag = 0;
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -342,7 +342,8 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         const bool seg_first = (i == 0) || cur.step == 0;
         const bool seg_last = (i + 1 == n_items) || cur.step == spt - 1;
         const int nch = min(CH, a.g.k_chunks - cur.step * CH);
-        if (!wait_warp(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 2)) break;
+        // the group that filled this A stage waited for the shared-memory stage (weights and activations)
+        // before it decoded, so its arrival also covers the activation tile
         if (!wait_warp(bar_afull + 8 * cur.astage, (uint32_t)cur.aphase, 3)) break;
         if (seg_first && !wait_warp(bar_accempty, (seg & 1u) ^ 1u, 4)) break;
         tc_fence_after();
@@ -383,7 +384,11 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     const bool issuer = GI && ((warp - 2) & 3) == 0;     // first warp of a group issues the group's MMAs
     uint32_t own_phase = 0, gseg = 0;                    // GI: parity of the group's A stage; segments seen
     bool fresh = true;                                   // GI: the group's accumulators hold nothing of this segment yet
-    const bool epi_warp = (group == 0);                  // warps 2..5 also run the epilogue
+    // Epilogue: with group issue only group 0 drains the (narrow) accumulators while the other groups
+    // keep decoding; otherwise every group drains its share of the columns of its TMEM lane quarter.
+    const bool epi_warp = !GI || (group == 0);
+    const int col_lo = GI ? 0 : group * (NT / GROUPS), col_hi = GI ? NT : col_lo + NT / GROUPS;
+    static_assert(GI || (NT / GROUPS) % 16 == 0, "epilogue column shares are multiples of 16");
     const bool leader = (threadIdx.x == 64);
     const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
     uint32_t seg = 0, epi_phase = 0;
@@ -503,7 +508,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         for (int q = 0; q < GROUPS; ++q) acc_valid[q] = (len >= GROUPS) || (((q - i0 % GROUPS + GROUPS) % GROUPS) < len);
       }
 #pragma unroll 1
-      for (int c0 = 0; c0 < NT; c0 += 16) {
+      for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
         uint32_t v[16];
         tc_ld16(tmem_base + lane_off + c0, v);
         tc_wait_ld();
@@ -557,7 +562,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       if (!epi_sync()) break;                                         // bcast may be rewritten after this
       if (!finisher) continue;
 #pragma unroll 1
-      for (int c0 = 0; c0 < NT; c0 += 16) {
+      for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
         float acc[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
