@@ -63,7 +63,7 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+                                          "-i", str(self.index), "-lms", "20"], stdout=f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -160,7 +160,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-extras", action="store_true", help="skip the skinny / prefill / W4A4 lines")
@@ -205,13 +205,27 @@ def main():
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
+    # The timed region replays a CUDA graph of the K steps (3 K kernel launches): the kernels run 10-25 us
+    # each, shorter than a Python-driven launch, and the metric is the device path.  The same steps launched
+    # one by one from the host are timed as well and reported as "stream_launch".
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    launches0 = b.razer_kernel_launches()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(args.steps):
+                step(i)
+    launches = b.razer_kernel_launches() - launches0      # kernels one replay executes
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
     if dist:
         dist.barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    launches0 = b.razer_kernel_launches()
-    ms = time_cuda(step, args.steps, torch)
-    launches = b.razer_kernel_launches() - launches0
+    ms = time_cuda(lambda i: graph.replay(), 1, torch) / args.steps
+    ms_stream = time_cuda(step, args.steps, torch)
     clocks = sampler.stop()
     if dist:
         t = torch.tensor([ms], device="cuda")
@@ -240,10 +254,22 @@ def main():
            "h2d_bytes_per_step": sum(2 * l["K"] for l in layers), "d2h_bytes_per_step": sum(2 * l["N"] for l in layers),
            "ms_per_step": ms_e2e}
 
+    def graph_time(fn, reps):
+        """ms per call of fn(i), i = 0..reps-1, replayed from a CUDA graph."""
+        g = torch.cuda.CUDAGraph()
+        s2 = torch.cuda.Stream()
+        s2.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s2):
+            with torch.cuda.graph(g, stream=s2):
+                for i in range(reps):
+                    fn(i)
+        torch.cuda.synchronize()
+        g.replay()
+        return time_cuda(lambda i: g.replay(), 3, torch) / reps
+
     per_shape = []
     for l in layers:
-        t = time_cuda(lambda i, l=l: b.razer_gemv(l["desc"], l["sets"][i % n_sets], l["x"], l["y"], l["ws"]),
-                      args.steps, torch)
+        t = graph_time(lambda i, l=l: b.razer_gemv(l["desc"], l["sets"][i % n_sets], l["x"], l["y"], l["ws"]), 4 * n_sets)
         gbs = algo_bytes(1, l["N"], l["K"]) / (t * 1e-3) / 1e9
         per_shape.append({"M": 1, "N": l["N"], "K": l["K"], "us": t * 1e3, "GBps": gbs, "frac_hbm": gbs / pk["hbm"]})
 
@@ -256,6 +282,8 @@ def main():
                    "l2": f"inputs larger than L2: weights rotate over {n_sets} packed copies, {packed_total / 1e6:.0f} MB",
                    "parallelism": "replicas" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "timing": "CUDA events around one replay of a CUDA graph holding the K steps",
+        "stream_launch": {"value": world * step_bytes / (ms_stream * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms_stream},
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": pk["hbm"], "unit": "GB/s",
                      "frac": value / world / pk["hbm"], "traffic": None, "peak_source": pk["source"],
                      "kernel": "razer_gemv (3 launches per step)", "algorithmic_bytes_per_step": step_bytes,
@@ -277,7 +305,7 @@ def main():
                 f = lambda i: b.razer_gemv(desc, sets[i % ns], x, y, ws)
                 for i in range(3):
                     f(i)
-                t = time_cuda(f, 30, torch)
+                t = graph_time(f, 4 * ns)
                 gbs = algo_bytes(M, N, K) / (t * 1e-3) / 1e9
                 extras.append({"config": 3, "op": "razer_gemv", "M": M, "N": N, "K": K, "us": t * 1e3, "GBps": gbs,
                                "frac_hbm": gbs / pk["hbm"], "TFLOPs": 2.0 * M * N * K / (t * 1e-3) / 1e12})
@@ -292,7 +320,7 @@ def main():
             f = lambda i: b.razer_gemm(desc, sets[i % 2], x, y, ws)
             for i in range(3):
                 f(i)
-            t = time_cuda(f, 10, torch)
+            t = graph_time(f, 8)
             tf = 2.0 * M * N * K / (t * 1e-3) / 1e12
             extras.append({"config": 4, "op": "razer_gemm", "M": M, "N": N, "K": K, "us": t * 1e3, "TFLOPs": tf,
                            "frac_bf16": tf / pk["bf16"]})
@@ -308,7 +336,7 @@ def main():
         f = lambda i: b.razer_gemm_w4a4(desc, sets[i % 4], ac, as_, ats, y=y, workspace=ws)
         for i in range(3):
             f(i)
-        t = time_cuda(f, 10, torch)
+        t = graph_time(f, 8)
         extras.append({"config": 5, "op": "razer_quant_act", "M": M, "K": K, "us": tq * 1e3,
                        "GBps": (M * K * 2 + M * K * 0.5625) / (tq * 1e-3) / 1e9})
         tf = 2.0 * M * N * K / (t * 1e-3) / 1e12
