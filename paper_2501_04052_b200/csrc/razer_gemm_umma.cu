@@ -279,7 +279,32 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x, THREADS);
+  // Producer state (thread 0 only).  The first ring of loads goes out before the rest of the prologue
+  // (tables, TMEM allocation) so that the first HBM round trip overlaps it.
+  int issued = 0;
+  int p_rt = cur.tile / a.token_tiles, p_tt = cur.tile - p_rt * a.token_tiles;
+  auto produce = [&]() {
+    const int c0 = cur.step * CH;
+    const int nch = min(CH, a.g.k_chunks - c0);
+    const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
+    const uint32_t bar = bar_full + 8 * cur.stage;
+    const uint32_t n_x = a.x_map_3d ? CH : nch;           // the 3-D box always spans CH chunks (zero-filled past K)
+    mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * Cfg::X_BOX_BYTES);
+    bulk_copy_g2s(st, a.packed + ((size_t)p_rt * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
+    if (a.x_map_3d) {
+      tma_load_3d(st + Cfg::W_PAD, &tmap_x, 0, p_tt * NT, c0, bar);
+    } else {
+      for (int c = 0; c < nch; ++c)
+        tma_load_2d(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, p_tt * NT, bar);
+    }
+    if (cur.step == spt - 1 && ++p_tt == a.token_tiles) { p_tt = 0; ++p_rt; }
+    cur.template next<STAGES, ASTAGES>(spt);
+  };
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    for (; issued < n_items && issued < STAGES; ++issued) produce();
+  }
+  if (warp != 0) decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x - 32, THREADS - 32);
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"((uint32_t)Cfg::TMEM_COLS)
@@ -300,26 +325,9 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
-      int issued = 0;
-      int rt = cur.tile / a.token_tiles, tt = cur.tile - rt * a.token_tiles;
       for (; issued < n_items; ++issued) {
         if (!mbar_wait(bar_empty + 8 * cur.stage, (uint32_t)cur.phase ^ 1u, abort_flag)) { fail(1); break; }
-        const int c0 = cur.step * CH;
-        const int nch = min(CH, a.g.k_chunks - c0);
-        const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
-        const uint32_t bar = bar_full + 8 * cur.stage;
-        const uint32_t n_x = a.x_map_3d ? CH : nch;       // the 3-D box always spans CH chunks (zero-filled past K)
-        mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * Cfg::X_BOX_BYTES);
-        bulk_copy_g2s(st, a.packed + ((size_t)rt * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
-        if (a.x_map_3d) {
-          tma_load_3d(st + Cfg::W_PAD, &tmap_x, 0, tt * NT, c0, bar);
-        } else {
-          for (int c = 0; c < nch; ++c)
-            tma_load_2d(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, tt * NT, bar);
-        }
-        if (cur.step == spt - 1 && ++tt == a.token_tiles) { tt = 0; ++rt; }
-        cur.template next<STAGES, ASTAGES>(spt);
+        produce();
       }
       // Drain: copies still in flight must land before this CTA's shared memory is released.
       const int pending = issued < STAGES ? issued : STAGES;
@@ -536,7 +544,8 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
           }
         } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) my_slot[(c0 + j) * TILE_ROWS + row] = __uint_as_float(v[j]);
+          for (int j = 0; j < 16; ++j)
+            if (m0 + c0 + j < a.M) my_slot[(c0 + j) * TILE_ROWS + row] = __uint_as_float(v[j]);
         }
       }
       tc_fence_before();
@@ -566,12 +575,24 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         float acc[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
-        for (int c = c_first; c <= c_last; ++c) {
-          const long long b_c = (a.total_items * c) / grid;
-          const int sl = (b_c / spt == tile) ? 0 : 1;
-          const float* src = a.slots + ((size_t)c * 2 + sl) * (size_t)(NT * TILE_ROWS);
+        const int m_valid = a.M - (m0 + c0);                           // tokens of this column group that exist
+        // ascending CTA order (a fixed summation order); the loads of two CTAs' slots are in flight together
+        for (int cb = c_first; cb <= c_last; cb += 2) {
+          float part[2][16];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) acc[j] += __ldcg(src + (c0 + j) * TILE_ROWS + row);
+          for (int u = 0; u < 2; ++u) {
+            const int c = cb + u;
+            const long long b_c = (a.total_items * (c <= c_last ? c : c_last)) / grid;
+            const int sl = (b_c / spt == tile) ? 0 : 1;
+            const float* src = a.slots + ((size_t)(c <= c_last ? c : c_last) * 2 + sl) * (size_t)(NT * TILE_ROWS);
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              part[u][j] = (c <= c_last && j < m_valid) ? __ldcg(src + (c0 + j) * TILE_ROWS + row) : 0.0f;
+          }
+#pragma unroll
+          for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int j = 0; j < 16; ++j) acc[j] += part[u][j];
         }
         if (n_out < a.g.N) {
 #pragma unroll

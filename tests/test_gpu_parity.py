@@ -251,3 +251,39 @@ def test_workspace_too_small_is_an_error(b):
         with pytest.raises(b.RazerError) as e:
             b.razer_gemv(desc, packed, x, workspace=tiny)
         assert e.value.code == b.ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ alternative kernels (chosen by environment)
+
+_ALT_KERNEL_CHECK = r"""
+import sys, numpy as np, torch
+sys.path.insert(0, sys.argv[1])
+from oracle import razer_oracle as ro
+from paper_2501_04052_b200 import binding as b, inputs
+for (M, N, K, seed) in [(1, 1000, 4160, 1), (5, 333, 2064, 2), (16, 640, 1024, 3)]:
+    codes, scales = inputs.random_codes(N, K, seed=seed, scale_lo=0, scale_hi=64, zero_block_frac=0.02)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc = b.make_desc(N, K, 0.004, sv_mag=(5.0, 9.0))
+    packed = b.razer_pack_layout(desc, torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda())
+    x = inputs.activations(M, K, seed)
+    ws = b.alloc_workspace(desc, M, b.OP_GEMV, "cuda")
+    y = b.razer_gemv(desc, packed, x.cuda(), workspace=ws)
+    b.razer_workspace_status(ws)
+    ref = ro.matmul_w4a16(inputs.bf16_to_bits(x), codes, scales, np.float32(0.004), sv_mag=(5.0, 9.0))
+    err = ro.rel_frobenius(inputs.bf16_to_bits(y.cpu()), ref)
+    assert err <= 1e-3, (M, N, K, err)
+print("ok")
+"""
+
+
+@pytest.mark.parametrize("kernel", ["mma", "simt"])
+def test_alternative_kernels_match_the_oracle(kernel):
+    """RAZER_KERNEL selects the register-fragment mma.sync kernel or the CUDA-core kernel for the same
+    entry point; the choice is read once per process, so the check runs in a child process."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, RAZER_KERNEL=kernel)
+    r = subprocess.run([sys.executable, "-c", _ALT_KERNEL_CHECK, root], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "ok" in r.stdout, r.stdout + r.stderr
