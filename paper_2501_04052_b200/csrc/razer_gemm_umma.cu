@@ -112,6 +112,12 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
   return pred != 0;
 }
+// Programmatic dependent launch: when the kernel was launched with the programmatic-serialization
+// attribute, `grid_dep_wait` returns once the preceding kernel in the stream has completed (otherwise at
+// once); everything that may depend on that kernel (activations, workspace, outputs) is touched after it,
+// while the weight stream, which depends on nothing, starts before.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -283,7 +289,19 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
   // (tables, TMEM allocation) so that the first HBM round trip overlaps it.
   int issued = 0;
   int p_rt = cur.tile / a.token_tiles, p_tt = cur.tile - p_rt * a.token_tiles;
-  auto produce = [&]() {
+  auto produce_x = [&](int stage, int step, int tt) {       // activation box(es) of one stage
+    const int c0 = step * CH;
+    const int nch = min(CH, a.g.k_chunks - c0);
+    const uint32_t st = smem_u32(smem) + (uint32_t)stage * Cfg::STAGE_BYTES;
+    const uint32_t bar = bar_full + 8 * stage;
+    if (a.x_map_3d) {
+      tma_load_3d(st + Cfg::W_PAD, &tmap_x, 0, tt * NT, c0, bar);
+    } else {
+      for (int c = 0; c < nch; ++c)
+        tma_load_2d(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, tt * NT, bar);
+    }
+  };
+  auto produce = [&](bool with_x) {
     const int c0 = cur.step * CH;
     const int nch = min(CH, a.g.k_chunks - c0);
     const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
@@ -291,18 +309,25 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     const uint32_t n_x = a.x_map_3d ? CH : nch;           // the 3-D box always spans CH chunks (zero-filled past K)
     mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * Cfg::X_BOX_BYTES);
     bulk_copy_g2s(st, a.packed + ((size_t)p_rt * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
-    if (a.x_map_3d) {
-      tma_load_3d(st + Cfg::W_PAD, &tmap_x, 0, p_tt * NT, c0, bar);
-    } else {
-      for (int c = 0; c < nch; ++c)
-        tma_load_2d(st + Cfg::W_PAD + c * Cfg::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, p_tt * NT, bar);
-    }
+    if (with_x) produce_x(cur.stage, cur.step, p_tt);
     if (cur.step == spt - 1 && ++p_tt == a.token_tiles) { p_tt = 0; ++p_rt; }
     cur.template next<STAGES, ASTAGES>(spt);
   };
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
-    for (; issued < n_items && issued < STAGES; ++issued) produce();
+    grid_dep_launch();                                    // the next kernel may start its own prologue
+    // first ring: packed weights now, their activation boxes once the preceding kernel has finished
+    const ItemCursor first = cur;
+    const int first_tt = p_tt;
+    for (; issued < n_items && issued < STAGES; ++issued) produce(false);
+    grid_dep_wait();
+    ItemCursor c2 = first;
+    int tt2 = first_tt;
+    for (int i = 0; i < issued; ++i) {
+      produce_x(c2.stage, c2.step, tt2);
+      if (c2.step == spt - 1 && ++tt2 == a.token_tiles) tt2 = 0;
+      c2.template next<STAGES, ASTAGES>(spt);
+    }
   }
   if (warp != 0) decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x - 32, THREADS - 32);
   if (warp == 1) {
@@ -319,6 +344,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
 
   auto fail = [&](uint32_t code) {
     *abort_flag = 1;
+    grid_dep_wait();                                      // the status word lives in the (possibly shared) workspace
     atomicCAS(a.status, 0u, code);
   };
 
@@ -327,7 +353,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     if (lane == 0) {
       for (; issued < n_items; ++issued) {
         if (!mbar_wait(bar_empty + 8 * cur.stage, (uint32_t)cur.phase ^ 1u, abort_flag)) { fail(1); break; }
-        produce();
+        produce(true);
       }
       // Drain: copies still in flight must land before this CTA's shared memory is released.
       const int pending = issued < STAGES ? issued : STAGES;
@@ -398,7 +424,8 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     const int col_lo = GI ? 0 : group * (NT / GROUPS), col_hi = GI ? NT : col_lo + NT / GROUPS;
     static_assert(GI || (NT / GROUPS) % 16 == 0, "epilogue column shares are multiples of 16");
     const bool leader = (threadIdx.x == 64);
-    const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
+    float ts = a.tensor_scale;                           // (x extra scale: read after the grid dependency)
+    bool dep_waited = false;
     uint32_t seg = 0, epi_phase = 0;
     // all 32 lanes take the same branch after a wait, so the .aligned tcgen05 instructions stay convergent
     auto wait_all = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
@@ -505,6 +532,11 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       const int rt = tile / a.token_tiles, tt = tile - rt * a.token_tiles;
       const int n_out = rt * TILE_ROWS + row;
       const int m0 = tt * NT;
+      if (!dep_waited) {                                   // outputs, workspace and the scale scalar may belong to the preceding kernel
+        grid_dep_wait();
+        if (a.extra_scale) ts *= *a.extra_scale;
+        dep_waited = true;
+      }
       if (!wait_all(bar_accfull, seg & 1u, 7)) break;
       tc_fence_after();
       const int slot_idx = (seg_begin == it_begin) ? 0 : 1;          // first segment of the stripe or not
@@ -699,9 +731,22 @@ static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, c
                          "cudaFuncSetAttribute(max dynamic shared memory)"));
     attr_set = true;
   }
-  kern<<<grid, 64 + 32 * NDW, Cfg::SMEM_BYTES, st>>>(tmap, args);
+  // Programmatic dependent launch (RAZER_PDL=0 turns it off): the kernel may begin while the preceding
+  // kernel of the stream drains; it touches nothing that kernel may own before its grid_dep_wait().
+  static const bool pdl = [] { const char* e = getenv("RAZER_PDL"); return !(e && e[0] == '0'); }();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(64 + 32 * NDW);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap, args);
   count_launches(1);
-  return check_cuda(cudaGetLastError(), "razer_umma_kernel launch");
+  return check_cuda(e, "razer_umma_kernel launch");
 }
 
 int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int M, int ldx_K, float extra_scale,
