@@ -585,17 +585,18 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       ++seg;
       if (complete) continue;
       // ---------------- partial tile: publish, count, last arrival reduces ----------------
-      __threadfence();
-      if (!epi_sync()) break;
+      if (!epi_sync()) break;                                         // all slot stores of this CTA are done (CTA scope)
       const int tile_end = tile_begin + spt;
       const int c_first = cta_of_item(tile_begin, grid, a.total_items);
       const int c_last = cta_of_item(tile_end - 1, grid, a.total_items);
       if (leader) {
         const uint32_t parts = (uint32_t)(c_last - c_first + 1);
-        const uint32_t prev = atomicAdd(a.counters + tile, 1u);
+        // release: the CTA's slot stores (ordered before this by the rendezvous) become visible with the count;
+        // acquire: the last arrival sees every earlier arrival's slot stores
+        uint32_t prev;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.counters + tile) : "memory");
         const uint32_t last = (prev + 1 == parts) ? 1u : 0u;
         if (last) a.counters[tile] = 0;                               // leave the counter ready for the next call
-        __threadfence();
         *bcast = last;
       }
       if (!epi_sync()) break;
@@ -688,8 +689,9 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  static const int ch16 = [] { const char* e = getenv("RAZER_CH"); return e ? atoi(e) : 4; }();   // tuning aid: 3 or 4
-  p.CH = p.NT == 16 ? (ch16 == 3 ? 3 : 4) : p.NT == 32 ? 4 : p.NT == 64 ? 2 : 1;
+  static const int ch16 = [] { const char* e = getenv("RAZER_CH"); return e ? atoi(e) : 0; }();   // tuning aid: 2, 3 or 4
+  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
+  if (p.NT == 16 && (ch16 == 2 || ch16 == 3)) p.CH = ch16;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -803,6 +805,7 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   switch (p.NT) {
     case 16:
       if (p.CH == 3) return launch_cfg<16, 3, 8, 4, 16, 4, true>(tmap, a, p.grid, st);
+      if (p.CH == 2) return launch_cfg<16, 2, 10, 3, 12, 6, true>(tmap, a, p.grid, st);
       return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
     case 32: return launch_cfg<32, 4, 5, 3, 12, 3, true>(tmap, a, p.grid, st);
     case 64: return launch_cfg<64, 2, 6, 4, 16, 4, true>(tmap, a, p.grid, st);

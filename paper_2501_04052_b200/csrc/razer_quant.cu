@@ -26,7 +26,16 @@ __global__ void act_amax_kernel(const uint4* __restrict__ x, long long n_vec, ui
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  if ((threadIdx.x & 31) == 0 && m) atomicMax(amax_bits, m);
+  // one atomic per CTA: thousands of atomics on one address would serialise in the L2
+  __shared__ uint32_t warp_max[32];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < (blockDim.x + 31) / 32 ? warp_max[threadIdx.x] : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (threadIdx.x == 0 && m) atomicMax(amax_bits, m);
+  }
 }
 
 // Round a non-negative finite float to the nearest E4M3 code (ties to even mantissa),
@@ -131,7 +140,11 @@ int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* sca
   };
   if (!scale_in) {
     RAZER_TRY(check_cuda(cudaMemsetAsync(amax_scratch, 0, sizeof(uint32_t), st), "amax memset"));
-    act_amax_kernel<<<grid(n_vec), threads, 0, st>>>((const uint4*)x, n_vec, amax_scratch);
+    {
+      long long b = (n_vec + threads * 4 - 1) / (threads * 4);        // four vectors per thread, at most two CTAs per SM
+      const int g2 = (int)(b < 1 ? 1 : (b > 296 ? 296 : b));
+      act_amax_kernel<<<g2, threads, 0, st>>>((const uint4*)x, n_vec, amax_scratch);
+    }
     count_launches(1);
     RAZER_TRY(check_cuda(cudaGetLastError(), "act_amax_kernel launch"));
   }
