@@ -415,7 +415,9 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     static_assert(NDW % 4 == 0 && GROUPS <= ASTAGES, "every dequant group needs an A stage of its own");
     static_assert(!GI || (NACC % GROUPS == 0 && ASTAGES == GROUPS), "group issue: A stage and accumulators per group");
     constexpr int APG = GI ? NACC / GROUPS : NACC;       // accumulators per group
-    const bool issuer = GI && ((warp - 2) & 3) == 0;     // first warp of a group issues the group's MMAs
+    // one warp of each group issues the group's MMAs; the groups pick different ones so that the issuing
+    // warps sit on different schedulers (a warp's scheduler is warp % 4)
+    const bool issuer = GI && ((warp - 2) & 3) == (group & 3);
     uint32_t own_phase = 0, gseg = 0;                    // GI: parity of the group's A stage; segments seen
     bool fresh = true;                                   // GI: the group's accumulators hold nothing of this segment yet
     // Epilogue: with group issue only group 0 drains the (narrow) accumulators while the other groups
