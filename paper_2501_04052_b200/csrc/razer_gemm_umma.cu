@@ -691,9 +691,7 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  static const int ch16 = [] { const char* e = getenv("RAZER_CH"); return e ? atoi(e) : 0; }();   // tuning aid: 2, 3 or 4
   p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
-  if (p.NT == 16 && (ch16 == 2 || ch16 == 3)) p.CH = ch16;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -806,8 +804,6 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   a.x_map_3d = map_3d;
   switch (p.NT) {
     case 16:
-      if (p.CH == 3) return launch_cfg<16, 3, 8, 4, 16, 4, true>(tmap, a, p.grid, st);
-      if (p.CH == 2) return launch_cfg<16, 2, 10, 3, 12, 6, true>(tmap, a, p.grid, st);
       return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
     case 32: return launch_cfg<32, 4, 5, 3, 12, 3, true>(tmap, a, p.grid, st);
     case 64: return launch_cfg<64, 2, 6, 4, 16, 4, true>(tmap, a, p.grid, st);
