@@ -35,7 +35,8 @@ namespace mma_path {
 
 constexpr uint32_t WAIT_LIMIT = 1u << 26;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
-constexpr int COMPUTE_WARPS = 8;
+constexpr int COMPUTE_WARPS = 16;
+constexpr int KQ = COMPUTE_WARPS / 4;                 // warps that share 32 rows split a stage's chunks KQ ways
 constexpr int THREADS = 32 * (1 + COMPUTE_WARPS);
 constexpr size_t WS_STATUS_BYTES = 256;
 
@@ -99,6 +100,8 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 // D (+)= A(16 x 16, row) * B(16 x 8, col), bf16 inputs, FP32 accumulation.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                           uint32_t b1) {
   asm volatile(
@@ -128,7 +131,7 @@ struct Cfg {
   static constexpr int X_BOX_BYTES = TOKENS * 128;               // tokens x 64 k x 2 B
   static constexpr int STAGE_BYTES = W_PAD + CH * X_BOX_BYTES;
   static constexpr int NUM_BARS = 2 * STAGES + 2;
-  static constexpr int RED_BYTES = TILE_ROWS * TOKENS * 4;       // partial sums of the odd-chunk warps
+  static constexpr int RED_BYTES = (KQ - 1) * TILE_ROWS * TOKENS * 4;   // partial sums of the warps with kq > 0
   static constexpr size_t SMEM_BYTES =
       1024 + (size_t)STAGES * STAGE_BYTES + RED_BYTES + DECODE_TABLE_BYTES + NUM_BARS * 8 + 64;
 };
@@ -179,34 +182,58 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
     flags[2] = 0;                                       // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x, THREADS);
-  __syncthreads();
-
   auto fail = [&](uint32_t code) {
     *abort_flag = 1;
+    grid_dep_wait();                                      // the status word lives in the (possibly shared) workspace
     atomicCAS(a.status, 0u, code);
   };
+  // Producer state (thread 0).  Weights depend on nothing and start at once; activation boxes wait for
+  // the preceding kernel of the stream (programmatic dependent launch).
+  int issued = 0;
+  auto produce_x = [&](int stg, int stp) {
+    const int c0 = stp * CH;
+    const int nch = min(CH, a.g.k_chunks - c0);
+    const uint32_t st = smem_u32(smem) + (uint32_t)stg * C::STAGE_BYTES;
+    const uint32_t bar = bar_full + 8 * stg;
+    if (a.x_map_3d) {
+      tma_load_3d(st + C::W_PAD, &tmap_x, 0, 0, c0, bar);
+    } else {
+      for (int c = 0; c < nch; ++c) tma_load_2d(st + C::W_PAD + c * C::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, 0, bar);
+    }
+  };
+  auto produce = [&](bool with_x) {
+    const int c0 = step * CH;
+    const int nch = min(CH, a.g.k_chunks - c0);
+    const uint32_t st = smem_u32(smem) + (uint32_t)stage * C::STAGE_BYTES;
+    const uint32_t bar = bar_full + 8 * stage;
+    const uint32_t n_x = a.x_map_3d ? CH : nch;           // the 3-D box always spans CH chunks (zero-filled past K)
+    mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * C::X_BOX_BYTES);
+    bulk_copy_g2s(st, a.packed + ((size_t)tile * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
+    if (with_x) produce_x(stage, step);
+    advance();
+  };
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    grid_dep_launch();
+    const int t0 = tile, s0 = step;
+    for (; issued < n_items && issued < STAGES; ++issued) produce(false);
+    grid_dep_wait();
+    int t2 = t0, s2 = s0;
+    for (int i = 0; i < issued; ++i) {
+      produce_x(i, s2);
+      if (++s2 == spt) { s2 = 0; ++t2; }
+    }
+    (void)t2;
+  }
+  if (warp != 0) decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x - 32, THREADS - 32);
+  __syncthreads();
 
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
-      int issued = 0;
       for (; issued < n_items; ++issued) {
         if (!mbar_wait(bar_empty + 8 * stage, (uint32_t)phase ^ 1u, abort_flag)) { fail(21); break; }
-        const int c0 = step * CH;
-        const int nch = min(CH, a.g.k_chunks - c0);
-        const uint32_t st = smem_u32(smem) + (uint32_t)stage * C::STAGE_BYTES;
-        const uint32_t bar = bar_full + 8 * stage;
-        const uint32_t n_x = a.x_map_3d ? CH : nch;       // the 3-D box always spans CH chunks (zero-filled past K)
-        mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * C::X_BOX_BYTES);
-        bulk_copy_g2s(st, a.packed + ((size_t)tile * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
-        if (a.x_map_3d) {
-          tma_load_3d(st + C::W_PAD, &tmap_x, 0, 0, c0, bar);
-        } else {
-          for (int c = 0; c < nch; ++c) tma_load_2d(st + C::W_PAD + c * C::X_BOX_BYTES, &tmap_x, (c0 + c) * CHUNK_K, 0, bar);
-        }
-        advance();
+        produce(true);
       }
       // Drain: copies still in flight must land before this CTA's shared memory is released.
       const int pending = issued < STAGES ? issued : STAGES;
@@ -216,13 +243,14 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
   } else {
     // ===================== compute warps =====================
     const int cw = warp - 1;
-    const int rg = cw & 3, half = cw >> 2;
+    const int rg = cw & 3, half = cw >> 2;              // half = kq: which share of the chunks
     const int g = lane >> 2, t = lane & 3;
     const bool epi_warp = (half == 0);
     const bool leader = (cw == 0 && lane == 0);
     const DecodeTables dt = decode_tables_view(tables, lane);
     const uint32_t mul_lo = a.mul_lo, mul_hi = a.mul_hi;
-    const float ts = a.extra_scale ? a.tensor_scale * *a.extra_scale : a.tensor_scale;
+    float ts = a.tensor_scale;                           // (x extra scale: read after the grid dependency)
+    bool dep_waited = false;
     uint32_t all_phase = 0, epi_phase = 0;
     auto wait_all = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
       const bool got = mbar_wait(bar, parity, abort_flag);
@@ -273,8 +301,8 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
       if (!wait_all(bar_full + 8 * stage, (uint32_t)phase, 24)) break;
       const uint32_t st = smem_addr(smem) + (uint32_t)stage * C::STAGE_BYTES;
 #pragma unroll
-      for (int cc = 0; cc < (CH + 1) / 2; ++cc) {
-        const int c = 2 * cc + half;
+      for (int cc = 0; cc < (CH + KQ - 1) / KQ; ++cc) {
+        const int c = KQ * cc + half;
         if (c < nch) {
           const uint32_t ck = st + c * CHUNK_BYTES;
           const uint32_t xk = st + C::W_PAD + c * C::X_BOX_BYTES;
@@ -313,7 +341,8 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
       const int tile_begin = tile * spt;
       const int seg_begin = it_begin > tile_begin ? it_begin : tile_begin;
       const bool complete = (seg_begin == tile_begin) && (step == spt - 1);
-      if (half == 1) {
+      if (half >= 1) {
+        float* red_w = red + (half - 1) * (TILE_ROWS * C::TOKENS);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -321,7 +350,7 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int r = 32 * rg + 16 * mt + 8 * (j >> 1) + g, m = 8 * nt + 2 * t + (j & 1);
-              red[m * TILE_ROWS + r] = acc[mt][nt][j];
+              red_w[m * TILE_ROWS + r] = acc[mt][nt][j];
               acc[mt][nt][j] = 0.0f;
             }
       }
@@ -334,11 +363,16 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int r = 32 * rg + 16 * mt + 8 * (j >> 1) + g, m = 8 * nt + 2 * t + (j & 1);
-              acc[mt][nt][j] += red[m * TILE_ROWS + r];
+              for (int q = 0; q < KQ - 1; ++q) acc[mt][nt][j] += red[q * (TILE_ROWS * C::TOKENS) + m * TILE_ROWS + r];
             }
       }
       if (!sync_all()) break;                               // `red` may be rewritten after this
       if (!epi_warp) continue;
+      if (!dep_waited) {                                   // outputs, workspace and the scale scalar may belong to the preceding kernel
+        grid_dep_wait();
+        if (a.extra_scale) ts *= *a.extra_scale;
+        dep_waited = true;
+      }
       const int slot_idx = (seg_begin == it_begin) ? 0 : 1;           // first segment of the stripe or not
       float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(C::TOKENS * TILE_ROWS);
 #pragma unroll
@@ -351,46 +385,71 @@ razer_mma_kernel(const __grid_constant__ CUtensorMap tmap_x, const Args a) {
             const int n_out = tile * TILE_ROWS + r;
             if (complete) {
               if (n_out < a.g.N && m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * acc[mt][nt][j]);
-            } else {
+            } else if (m < a.M) {
               my_slot[m * TILE_ROWS + r] = acc[mt][nt][j];
             }
             acc[mt][nt][j] = 0.0f;
           }
       if (complete) continue;
       // ---------------- partial tile: publish, count, last arrival reduces ----------------
-      __threadfence();
-      if (!sync_epi()) break;
+      if (!sync_epi()) break;                                         // all slot stores of this CTA are done (CTA scope)
       const int tile_end = tile_begin + spt;
       const int c_first = cta_of_item(tile_begin, grid, a.total_items);
       const int c_last = cta_of_item(tile_end - 1, grid, a.total_items);
       if (leader) {
         const uint32_t parts = (uint32_t)(c_last - c_first + 1);
-        const uint32_t prev = atomicAdd(a.counters + tile, 1u);
+        // release: the CTA's slot stores become visible with the count; acquire: the last arrival sees all of them
+        uint32_t prev;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.counters + tile) : "memory");
         const uint32_t last = (prev + 1 == parts) ? 1u : 0u;
         if (last) a.counters[tile] = 0;                               // leave the counter ready for the next call
-        __threadfence();
         *bcast = last;
       }
       if (!sync_epi()) break;
       const bool finisher = *reinterpret_cast<volatile uint32_t*>(bcast) != 0;
       if (!sync_epi()) break;                                         // bcast may be rewritten after this
       if (!finisher) continue;
+      {
+        float sum[2][NTILES][4];
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
+        for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < NTILES; ++nt)
+          for (int nt = 0; nt < NTILES; ++nt)
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int r = 32 * rg + 16 * mt + 8 * (j >> 1) + g, m = 8 * nt + 2 * t + (j & 1);
-            const int n_out = tile * TILE_ROWS + r;
-            float sum = 0.0f;
-            for (int c = c_first; c <= c_last; ++c) {                  // ascending CTA order: a fixed summation order
-              const long long b_c = ((long long)a.total_items * c) / grid;
-              const int sl = (b_c / spt == tile) ? 0 : 1;
-              sum += __ldcg(a.slots + ((size_t)c * 2 + sl) * (size_t)(C::TOKENS * TILE_ROWS) + m * TILE_ROWS + r);
+            for (int j = 0; j < 4; ++j) sum[mt][nt][j] = 0.0f;
+        // ascending CTA order (a fixed summation order); all of a CTA's values are loaded before they are added
+        for (int c = c_first; c <= c_last; ++c) {
+          const long long b_c = ((long long)a.total_items * c) / grid;
+          const int sl = (b_c / spt == tile) ? 0 : 1;
+          const float* src = a.slots + ((size_t)c * 2 + sl) * (size_t)(C::TOKENS * TILE_ROWS);
+          float part[2][NTILES][4];
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTILES; ++nt)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int r = 32 * rg + 16 * mt + 8 * (j >> 1) + g, m = 8 * nt + 2 * t + (j & 1);
+                part[mt][nt][j] = (m < a.M) ? __ldcg(src + m * TILE_ROWS + r) : 0.0f;
+              }
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTILES; ++nt)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) sum[mt][nt][j] += part[mt][nt][j];
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NTILES; ++nt)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int r = 32 * rg + 16 * mt + 8 * (j >> 1) + g, m = 8 * nt + 2 * t + (j & 1);
+              const int n_out = tile * TILE_ROWS + r;
+              if (n_out < a.g.N && m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * sum[mt][nt][j]);
             }
-            if (n_out < a.g.N && m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * sum);
-          }
+      }
       (void)it;
     }
   }
@@ -474,9 +533,20 @@ static int mma_launch_cfg(const CUtensorMap& tmap, const mma_path::Args& args, i
                          "cudaFuncSetAttribute(max dynamic shared memory)"));
     attr_set = true;
   }
-  kern<<<grid, mma_path::THREADS, C::SMEM_BYTES, st>>>(tmap, args);
+  static const bool pdl = [] { const char* e = getenv("RAZER_PDL"); return !(e && e[0] == '0'); }();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(mma_path::THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap, args);
   count_launches(1);
-  return check_cuda(cudaGetLastError(), "razer_mma_kernel launch");
+  return check_cuda(e, "razer_mma_kernel launch");
 }
 
 int launch_gemv_mma(const razer_desc* d, const void* packed, const void* x, int M, float extra_scale,
