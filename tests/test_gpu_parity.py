@@ -287,3 +287,36 @@ def test_alternative_kernels_match_the_oracle(kernel):
     env = dict(os.environ, RAZER_KERNEL=kernel)
     r = subprocess.run([sys.executable, "-c", _ALT_KERNEL_CHECK, root], env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "ok" in r.stdout, r.stdout + r.stderr
+
+
+def test_back_to_back_dependent_launches(b):
+    """The matmul kernels start their weight stream while the preceding kernel of the stream still runs
+    (programmatic dependent launch) and must read activations, workspace and outputs only after it has
+    finished.  A chain y1 = W1 x, y2 = W2 y1, y3 = W1 y2 with shared workspace, launched back to back many
+    times, is compared with the same chain computed by the oracle."""
+    N = K = 2048
+    M = 3
+    c1, s1 = inputs.random_codes(N, K, seed=131)
+    c2, s2 = inputs.random_codes(N, K, seed=132)
+    c1, s1, c2, s2 = c1.numpy(), s1.numpy(), c2.numpy(), s2.numpy()
+    d1, p1 = _pack(b, c1, s1, 0.002)
+    d2, p2 = _pack(b, c2, s2, 0.002)
+    x = inputs.activations(M, K, 133)
+    ws = b.alloc_workspace(d1, M, b.OP_GEMV, "cuda")
+    xd = x.cuda()
+    bufs = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    outs = []
+    for rep in range(20):
+        b.razer_gemv(d1, p1, xd, bufs[0], ws)
+        b.razer_gemv(d2, p2, bufs[0], bufs[1], ws)
+        b.razer_gemv(d1, p1, bufs[1], bufs[2], ws)
+        outs.append(bufs[2].clone())
+    b.razer_workspace_status(ws)
+    y1 = ro.matmul_w4a16(inputs.bf16_to_bits(x), c1, s1, np.float32(0.002))
+    y2 = ro.matmul_w4a16(y1, c2, s2, np.float32(0.002))
+    y3 = ro.matmul_w4a16(y2, c1, s1, np.float32(0.002))
+    for o in outs:
+        assert torch.equal(o, outs[0]), "a repetition of the chain differs"
+    # three chained bf16 roundings: allow a few times the single-product bar
+    assert rel_fro_bits(outs[0], y3) <= 5e-3
+    assert rel_fro_bits(bufs[0], y1) <= TOL
