@@ -77,6 +77,10 @@ int launch_gemv_mma(const razer_desc*, const void* packed, const void* x, int M,
                     const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
 size_t gemv_mma_workspace_bytes(const razer_desc*, int M);
 bool gemv_mma_supported(const razer_desc*, int M);
+int launch_gemv_direct(const razer_desc*, const void* packed, const void* x, int M, float extra_scale,
+                       const float* extra_scale_dev, void* y, cudaStream_t);
+bool gemv_direct_supported(const razer_desc*, int M);
+double gemv_direct_balance(const razer_desc*);
 
 // Kernel choice: the tcgen05 kernel serves every M.  RAZER_KERNEL=mma (environment) routes M <= 16 to the
 // register-fragment mma.sync kernel instead (kept for comparison: it measures slower on B200), =simt routes
@@ -86,6 +90,7 @@ static char kernel_override() {
   return c;
 }
 static bool use_mma(const razer_desc* d, int M) { return kernel_override() == 'm' && gemv_mma_supported(d, M); }
+static bool use_direct(const razer_desc* d, int M) { return kernel_override() == 'd' && gemv_direct_supported(d, M); }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -176,6 +181,8 @@ static int matmul_common(const razer_desc* d, const void* packed_dev, const void
   RAZER_TRY(check_ptr(y_dev, 2, "y_dev"));
   if (ws && reinterpret_cast<uintptr_t>(ws) % 256)
     return set_error(RAZER_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+  if (use_direct(d, M))
+    return launch_gemv_direct(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, st);
   if (use_mma(d, M))
     return launch_gemv_mma(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   if (umma_supported(d, M))
