@@ -82,17 +82,36 @@ int launch_gemv_direct(const razer_desc*, const void* packed, const void* x, int
 bool gemv_direct_supported(const razer_desc*, int M);
 double gemv_direct_balance(const razer_desc*);
 
-// Kernel choice: the tcgen05 kernel serves every M.  RAZER_KERNEL=mma (environment) routes M <= 16 to the
-// register-fragment mma.sync kernel instead (kept for comparison: it measures slower on B200), =simt routes
-// everything to the CUDA-core kernel (debugging aid).
+// Kernel choice.  The tcgen05 kernel serves every M.  For M <= 8 the register-fragment kernel without split-K
+// (razer_gemv_direct.cu) is faster whenever its fixed cost matters or the rows divide well over the SMs
+// (measured on B200: 5.8 against 12.7 us for 4096 x 4096, level at 132 MB with 28672 rows, behind at 132 MB with
+// 8192 rows), so it takes those shapes.  RAZER_KERNEL (environment, read once) overrides: "umma" keeps
+// everything on the tcgen05 kernel, "direct" takes the register kernel wherever it is able to run, "mma"
+// routes M <= 16 to the older ring-fed mma.sync kernel (kept for comparison), "simt" routes everything to
+// the CUDA-core kernel (debugging aid).
 static char kernel_override() {
   static const char c = [] { const char* e = getenv("RAZER_KERNEL"); return e ? e[0] : '\0'; }();
   return c;
 }
 static bool use_mma(const razer_desc* d, int M) { return kernel_override() == 'm' && gemv_mma_supported(d, M); }
-static bool use_direct(const razer_desc* d, int M) { return kernel_override() == 'd' && gemv_direct_supported(d, M); }
+static bool use_direct(const razer_desc* d, int M) {
+  const char o = kernel_override();
+  if (!gemv_direct_supported(d, M)) return false;
+  if (o == 'd') return true;
+  if (o != '\0') return false;
+  const size_t bytes = make_geometry(d->N, d->K).packed_bytes();
+  return bytes <= ((size_t)64 << 20) || gemv_direct_balance(d) >= 0.9;
+}
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Workspace of a matmul against M tokens: enough for whichever kernel takes the shape.
+static size_t matmul_workspace_need(const razer_desc* d, int M) {
+  size_t b = simt_workspace_bytes(d, M);
+  if (umma_supported(d, M)) b = b > umma_workspace_bytes(d, M) ? b : umma_workspace_bytes(d, M);
+  if (gemv_mma_supported(d, M)) b = b > gemv_mma_workspace_bytes(d, M) ? b : gemv_mma_workspace_bytes(d, M);
+  return b;
+}
 
 }  // namespace razer
 
@@ -139,14 +158,10 @@ int razer_workspace_bytes(const razer_desc* d, int M, int op, size_t* bytes_out)
       if (M > 64) return set_error(RAZER_ERR_INVALID_ARG, "razer_gemv takes 1 <= M <= 64 (got %d)", M);
       /* fall through */
     case RAZER_OP_GEMM:
-      b = simt_workspace_bytes(d, M);
-      if (umma_supported(d, M)) b = b > umma_workspace_bytes(d, M) ? b : umma_workspace_bytes(d, M);
-      if (gemv_mma_supported(d, M)) b = b > gemv_mma_workspace_bytes(d, M) ? b : gemv_mma_workspace_bytes(d, M);
+      b = matmul_workspace_need(d, M);
       break;
     case RAZER_OP_GEMM_W4A4: {
-      size_t g = simt_workspace_bytes(d, M);
-      if (umma_supported(d, M)) g = g > umma_workspace_bytes(d, M) ? g : umma_workspace_bytes(d, M);
-      if (gemv_mma_supported(d, M)) g = g > gemv_mma_workspace_bytes(d, M) ? g : gemv_mma_workspace_bytes(d, M);
+      const size_t g = matmul_workspace_need(d, M);
       b = align_up((size_t)M * d->K * 2, 256) + g;
       break;
     }
@@ -181,8 +196,13 @@ static int matmul_common(const razer_desc* d, const void* packed_dev, const void
   RAZER_TRY(check_ptr(y_dev, 2, "y_dev"));
   if (ws && reinterpret_cast<uintptr_t>(ws) % 256)
     return set_error(RAZER_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
-  if (use_direct(d, M))
+  if (use_direct(d, M)) {
+    // this kernel needs no scratch, but the contract (a workspace of razer_workspace_bytes) is the same for every shape
+    const size_t need = matmul_workspace_need(d, M);
+    if (!ws || ws_bytes < need)
+      return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
     return launch_gemv_direct(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, st);
+  }
   if (use_mma(d, M))
     return launch_gemv_mma(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   if (umma_supported(d, M))

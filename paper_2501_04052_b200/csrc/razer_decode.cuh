@@ -99,6 +99,18 @@ __device__ __forceinline__ void decode_block_consts_byte(const DecodeTables& t, 
   svc.pad = 0;
 }
 
+// The same for a scale word rotated so that the block's byte sits on bits 14:7 (higher and lower bits may hold
+// anything), for tables that start on a 16 KB boundary of the shared window: the table offsets are then
+// merged into the addresses by the same logic op that isolates them.
+__device__ __forceinline__ void decode_block_consts_rot(const DecodeTables& t, uint32_t r, uint32_t& ss2, SvConsts& svc) {
+  ss2 = lds32(and_or(r, 0x3F80u, t.ss_lane));
+  const uint4 c = lds128(and_or(r >> 10, 0x10u, t.sv));
+  svc.sv = c.x;
+  svc.nsv_lo = c.y;
+  svc.nsv_hi = c.z;
+  svc.pad = 0;
+}
+
 // Four stored nibbles of each 16-bit half of `w` -> four bf16x2 registers (elements 2p, 2p+1
 // of the word in register p), each the exact product value x scale with the block's sign.
 // mul_lo = 2^6 + 2^12, mul_hi = 2^2 + 2^8 (run-time values so that they stay multiplies).

@@ -31,32 +31,35 @@ namespace direct_path {
 constexpr int WARPS = 16;
 constexpr int THREADS = 32 * WARPS;
 constexpr int TOKENS = 8;
-constexpr int DEPTH_MT1 = 5;    // chunks in flight per warp (register sets)
-constexpr int DEPTH_MT2 = 3;
+constexpr int UNIT_ROWS = 32;                       // two 16-row MMA tiles
+constexpr int DEPTH = 4;                            // chunk slices in flight per warp
+// A warp's ring stage: the 32-row slice of one chunk, [blk 0..3][32 slots x 8 B] (blocks 2 and 3 sit 32 bytes
+// further so that a half-warp's 8-byte reads, four blocks x four slots, cover all 32 banks), then
+// [32 rows x 4 scale bytes], then the activations of the chunk: lane l keeps its 16 columns (token l / 4,
+// columns 16 (l % 4) ..) as two 16-byte halves at 16 l and 512 + 16 l.
+constexpr int STAGE_CODE_BYTES = 4 * 256 + 32;
+constexpr int STAGE_X_OFF = STAGE_CODE_BYTES + 128;
+constexpr int STAGE_BYTES = STAGE_X_OFF + 1024;
+constexpr int RED_FLOATS = UNIT_ROWS * TOKENS;      // one warp's partial sums
+constexpr int RED_BYTES = 2 * WARPS * RED_FLOATS * 4;
+constexpr int RING_BYTES = WARPS * DEPTH * STAGE_BYTES;
+constexpr int TABLE_ALIGN = 16384;                  // decode_block_consts_rot() wants the tables on a 16 KB boundary
+constexpr size_t SMEM_BYTES = TABLE_ALIGN + DECODE_TABLE_BYTES + RING_BYTES + RED_BYTES;
+static_assert(STAGE_BYTES % 16 == 0 && STAGE_X_OFF % 16 == 0 && DECODE_TABLE_BYTES % 16 == 0, "16-byte copies");
+constexpr long long STEP_BYTES = (long long)WARPS * CHUNK_BYTES;   // a warp's next chunk of the same unit
 
-template <int MT>
-struct Cfg {
-  static constexpr int R = 16 * MT;                               // rows of a unit
-  static constexpr int RED_FLOATS = R * TOKENS;                   // one warp's partial sums
-  static constexpr int RED_BYTES = 2 * WARPS * RED_FLOATS * 4;    // two buffers
-  static constexpr size_t SMEM_BYTES = RED_BYTES + DECODE_TABLE_BYTES;
-};
+__device__ __forceinline__ constexpr int stage_blk_off(int blk) { return blk * 256 + (blk >> 1) * 32; }
 
-__device__ __forceinline__ uint2 ldg_stream64(const void* p) {
-  uint2 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
-  return v;
+// 16 bytes, of which only the first `bytes` (0 or 16) are read; the rest is written as zero
+__device__ __forceinline__ void cp_async16_cg(uint32_t dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ uint32_t ldg_stream32(const void* p) {
-  uint32_t v;
-  asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-  return v;
+__device__ __forceinline__ void cp_async16_ca(uint32_t dst, const void* src, uint32_t bytes) {   // kept in L1: re-read per unit
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ uint4 ldg128(const void* p) {   // activations: cached, re-read for every unit
-  uint4 v;
-  asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 // D (+)= A(16 x 16, row) * B(16 x 8, col), bf16 inputs, FP32 accumulation.
@@ -76,85 +79,134 @@ struct Args {
   Geometry g;
   float sv0, sv1, tensor_scale;
   uint32_t mul_lo, mul_hi;   // 2^6 + 2^12 and 2^2 + 2^8 (razer_decode.cuh)
-  int M, units;              // units of R rows
+  int M, halves;             // 16-row half units of the padded matrix
+  int unit_aligned;          // every CTA owns whole 32-row units (grid = units)
 };
 
-// One chunk's registers of a lane: code words and scale words of rows (g, g + 8) of each MMA tile,
-// and the lane's 16 activation columns (token g).
-template <int MT>
-struct ChunkRegs {
-  uint2 cw[MT][2];
-  uint32_t sw[MT][2];
-  uint4 xa, xb;
-};
+// One chunk slice of one MMA tile (16 rows): decode the lane's two blocks, four MMAs.
+// rot = (8 t + 25) % 32 turns the row's scale word so that block t's byte sits on bits 14:7.
+__device__ __forceinline__ void tile_step(float (&acc)[4], uint32_t st_codes, uint32_t st_scales, uint32_t rot,
+                                          const DecodeTables& dt, uint32_t mul_lo, uint32_t mul_hi,
+                                          const uint32_t (&xq)[4][2], uint32_t off_h0, uint32_t off_h1) {
+  const uint2 c0 = lds64(st_codes + off_h0), c1 = lds64(st_codes + off_h1);
+  const uint32_t s0 = lds32(st_scales), s1 = lds32(st_scales + 32);
+  uint32_t e[2][8];
+  {
+    uint32_t ss2;
+    SvConsts svc;
+    decode_block_consts_rot(dt, __funnelshift_r(s0, s0, rot), ss2, svc);
+    decode_word(c0.x, ss2, svc, mul_lo, mul_hi, e[0]);
+    decode_word(c0.y, ss2, svc, mul_lo, mul_hi, e[0] + 4);
+  }
+  {
+    uint32_t ss2;
+    SvConsts svc;
+    decode_block_consts_rot(dt, __funnelshift_r(s1, s1, rot), ss2, svc);
+    decode_word(c1.x, ss2, svc, mul_lo, mul_hi, e[1]);
+    decode_word(c1.y, ss2, svc, mul_lo, mul_hi, e[1] + 4);
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    mma_16816(acc, e[0][2 * q], e[1][2 * q], e[0][2 * q + 1], e[1][2 * q + 1], xq[q][0], xq[q][1]);
+}
 
-template <int MT, int DEPTH>
 __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) {
-  using C = Cfg<MT>;
-  extern __shared__ __align__(16) uint8_t smem[];
-  float* red = reinterpret_cast<float*>(smem);
-  uint8_t* tables = smem + C::RED_BYTES;
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  // tables first, on a 16 KB boundary of the shared window; then the rings; then the reduction buffers
+  const uint32_t raw_addr = smem_addr(smem_raw);
+  uint8_t* tables = smem_raw + (((raw_addr + TABLE_ALIGN - 1) & ~(uint32_t)(TABLE_ALIGN - 1)) - raw_addr);
+  uint8_t* ring_base = tables + DECODE_TABLE_BYTES;
+  float* red = reinterpret_cast<float*>(ring_base + RING_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int kc = a.g.k_chunks;                               // >= WARPS (host check): every warp has chunks
-  const int u_begin = (int)(((long long)a.units * blockIdx.x) / gridDim.x);
-  const int u_end = (int)(((long long)a.units * (blockIdx.x + 1)) / gridDim.x);
+  const int per_unit = (kc - warp + WARPS - 1) / WARPS;      // this warp's chunks of a unit: warp, warp + 16, ...
+  // this CTA's rows: a contiguous range of 16-row halves; a 32-row unit at either end may be shared with a neighbour
+  int h_begin, h_end;
+  if (a.unit_aligned) {
+    h_begin = 2 * blockIdx.x;
+    h_end = min(h_begin + 2, a.halves);
+  } else {
+    h_begin = (int)(((long long)a.halves * blockIdx.x) / gridDim.x);
+    h_end = (int)(((long long)a.halves * (blockIdx.x + 1)) / gridDim.x);
+  }
+  const int u_begin = h_begin >> 1, u_end = (h_end + 1) >> 1;
+  auto unit_mask = [&](int u) -> uint32_t {                  // which MMA tiles of unit u are this CTA's
+    return (2 * u >= h_begin && 2 * u < h_end ? 1u : 0u) | (2 * u + 1 >= h_begin && 2 * u + 1 < h_end ? 2u : 0u);
+  };
 
   grid_dep_launch();
   decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x, THREADS);
 
-  // this lane's byte offsets inside a chunk, relative to the unit's first row
-  int code_off[MT][2], scale_off[MT][2];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int r = 16 * mt + 8 * h + g;                     // units start on multiples of 16 rows: the slot swizzle stays inside
-      code_off[mt][h] = packed_code_offset(t, r);
-      scale_off[mt][h] = CHUNK_CODE_BYTES + r * 4;
-    }
+  const uint32_t ring = smem_addr(ring_base) + (uint32_t)warp * (DEPTH * STAGE_BYTES);
   const bool has_token = g < a.M;
-  const __nv_bfloat16* x_lane = a.x + (size_t)(has_token ? g : 0) * a.g.K + 16 * t;
-
-  auto load_w = [&](ChunkRegs<MT>& r, int u, int c) {       // weights: no dependency on earlier kernels
-    const int n0 = u * C::R, tile = n0 / TILE_ROWS, r0 = n0 % TILE_ROWS;
-    const uint8_t* ck = a.packed + ((size_t)tile * kc + c) * CHUNK_BYTES;
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        r.cw[mt][h] = ldg_stream64(ck + r0 * 8 + code_off[mt][h]);
-        r.sw[mt][h] = ldg_stream32(ck + r0 * 4 + scale_off[mt][h]);
-      }
+  // ---- copy side: what this lane copies for every chunk slice ----
+  // two 16-byte pieces of code words (blocks cblk and cblk + 2, slots 2 piece and + 1), 16 bytes of scale
+  // words (lanes 0..7) and its own 32 bytes of activations; a size of 0 writes zeros and reads nothing
+  const int piece = lane & 15, cblk = lane >> 4;
+  const uint32_t dst_codes = ring + stage_blk_off(cblk) + piece * 16;       // blocks cblk + 2: 544 bytes further
+  const uint32_t dst_lane = ring + lane * 16;                                 // + STAGE_CODE_BYTES: scales, + STAGE_X_OFF: activations
+  const uint8_t* src_codes;                                                   // blocks cblk + 2: 2048 bytes further
+  const uint8_t* src_scales;
+  const __nv_bfloat16* src_x;
+  int col, cp_unit, cp_left;                                                  // first activation column; unit; chunks of it still to copy
+  uint32_t sz_codes, sz_scales;
+  auto cursor_to_unit = [&](int u) {
+    const int n0 = u * UNIT_ROWS, tile = n0 / TILE_ROWS, r0 = n0 % TILE_ROWS;
+    const uint8_t* ck = a.packed + ((size_t)tile * kc + warp) * CHUNK_BYTES;
+    const uint32_t mask = u < u_end ? unit_mask(u) : 0u;
+    src_codes = ck + r0 * 8 + cblk * 1024 + piece * 16;
+    src_scales = ck + CHUNK_CODE_BYTES + r0 * 4 + (lane & 7) * 16;
+    src_x = a.x + (size_t)(has_token ? g : 0) * a.g.K + warp * CHUNK_K + 16 * t;
+    col = warp * CHUNK_K + 16 * t;
+    cp_unit = u;
+    cp_left = per_unit;
+    sz_codes = ((mask >> (piece >> 3)) & 1u) ? 16u : 0u;
+    sz_scales = ((mask >> ((lane & 7) >> 2)) & 1u) ? 16u : 0u;
   };
-  auto load_x = [&](ChunkRegs<MT>& r, int c) {
-    if (has_token && c * CHUNK_K + 16 * t < a.g.K) {         // K is a multiple of 16: a 16-column group is whole
-      r.xa = ldg128(x_lane + (size_t)c * CHUNK_K);
-      r.xb = ldg128(x_lane + (size_t)c * CHUNK_K + 8);
+  auto copy_weights = [&](uint32_t so) {                     // weights: no dependency on earlier kernels
+    if (cp_unit < u_end) {
+      cp_async16_cg(dst_codes + so, src_codes, sz_codes);
+      cp_async16_cg(dst_codes + so + 544, src_codes + 2048, sz_codes);
+      if (lane < 8) cp_async16_cg(dst_lane + so + STAGE_CODE_BYTES, src_scales, sz_scales);
+    }
+  };
+  auto copy_x = [&](uint32_t so) {
+    if (has_token && cp_unit < u_end) {
+      const bool in = col < a.g.K;                           // K is a multiple of 16: a 16-column group is whole
+      const __nv_bfloat16* src = in ? src_x : a.x;
+      cp_async16_ca(dst_lane + so + STAGE_X_OFF, src, in ? 16u : 0u);
+      cp_async16_ca(dst_lane + so + STAGE_X_OFF + 512, src + 8, in ? 16u : 0u);
+    }
+  };
+  auto cursor_next = [&]() {
+    if (--cp_left > 0) {
+      src_codes += STEP_BYTES;
+      src_scales += STEP_BYTES;
+      src_x += WARPS * CHUNK_K;
+      col += WARPS * CHUNK_K;
     } else {
-      r.xa = make_uint4(0, 0, 0, 0);
-      r.xb = make_uint4(0, 0, 0, 0);
-    }
-  };
-  auto advance = [&](int& u, int& c) {
-    c += WARPS;
-    if (c >= kc) {
-      c = warp;
-      ++u;
+      cursor_to_unit(cp_unit + 1);
     }
   };
 
-  // ---------------- prologue: the first DEPTH chunks' weights, then (after the dependency) their activations ----------------
-  ChunkRegs<MT> regs[DEPTH];
-  int pu = u_begin, pc = warp;                               // prefetch cursor
-  {
-    int u = pu, c = pc;
+  // lanes without a token never copy activations: their slots stay zero
+  if (!has_token) {
+    uint8_t* mine = ring_base + (size_t)warp * (DEPTH * STAGE_BYTES) + STAGE_X_OFF + lane * 16;
 #pragma unroll
     for (int d = 0; d < DEPTH; ++d) {
-      if (u < u_end) load_w(regs[d], u, c);
-      advance(u, c);
+      *reinterpret_cast<uint4*>(mine + d * STAGE_BYTES) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(mine + d * STAGE_BYTES + 512) = make_uint4(0, 0, 0, 0);
     }
+  }
+
+  // ---------------- prologue: the first DEPTH slices' weights, then (after the dependency) their activations ----------------
+  cursor_to_unit(u_begin);
+#pragma unroll
+  for (int d = 0; d < DEPTH; ++d) {
+    copy_weights(d * STAGE_BYTES);
+    cursor_next();
   }
   __syncthreads();                                           // tables are ready
   const DecodeTables dt = decode_tables_view(tables, lane);
@@ -162,79 +214,68 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   grid_dep_wait();                                           // activations and outputs may belong to the preceding kernel
   float ts = a.tensor_scale;
   if (a.extra_scale) ts *= *a.extra_scale;
+  cursor_to_unit(u_begin);
 #pragma unroll
   for (int d = 0; d < DEPTH; ++d) {
-    if (pu < u_end) load_x(regs[d], pc);
-    advance(pu, pc);
+    copy_x(d * STAGE_BYTES);
+    cp_async_commit();                                       // one group per position (the first also holds all the weights above)
+    cursor_next();
   }
 
-  float acc[MT][4];
+  // ---- compute side: this lane's reads from a stage ----
+  const uint32_t lo = (t & 1) ? 64u : 0u;                    // odd blocks keep rows g and g + 8 the other way round
+  const uint32_t rd_codes = ring + stage_blk_off(t) + g * 8;
+  const uint32_t rd_scales = ring + STAGE_CODE_BYTES + g * 4;
+  const uint32_t rot = (uint32_t)(8 * t + 25) & 31u;
+  float acc[2][4];
 #pragma unroll
-  for (int mt = 0; mt < MT; ++mt)
+  for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[mt][j] = 0.0f;
 
-  auto compute = [&](const ChunkRegs<MT>& r) {
-    const uint32_t xq[4][2] = {{r.xa.x, r.xa.y}, {r.xa.z, r.xa.w}, {r.xb.x, r.xb.y}, {r.xb.z, r.xb.w}};
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-      uint32_t e[2][8];
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint32_t ss2;
-        SvConsts svc;
-        decode_block_consts_byte(dt, r.sw[mt][h] >> (8 * t), ss2, svc);
-        decode_word(r.cw[mt][h].x, ss2, svc, mul_lo, mul_hi, e[h]);
-        decode_word(r.cw[mt][h].y, ss2, svc, mul_lo, mul_hi, e[h] + 4);
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        mma_16816(acc[mt], e[0][2 * q], e[1][2 * q], e[0][2 * q + 1], e[1][2 * q + 1], xq[q][0], xq[q][1]);
-    }
-  };
-
-  // End of a unit: leave this warp's partial sums, meet, and let R * 8 threads finish the rows.
-  // Element (row, token) of the unit sits at row * 8 + token, so a warp's 32 stores hit 32 banks.
+  uint32_t so = 0;                                           // byte offset of the current stage in the ring
   int buf = 0;
-  auto unit_end = [&](int u) {
-    float* mine = red + (buf * WARPS + warp) * C::RED_FLOATS;
+  for (int u = u_begin; u < u_end; ++u) {
+    const uint32_t mask = unit_mask(u);
+#pragma unroll 1
+    for (int j = 0; j < per_unit; ++j) {
+      cp_async_wait<DEPTH - 1>();                            // this lane's pieces of the oldest slice have landed
+      __syncwarp();                                          // ... and so have the other lanes'
+      const uint4 xa = lds128(dst_lane + so + STAGE_X_OFF), xb = lds128(dst_lane + so + STAGE_X_OFF + 512);
+      const uint32_t xq[4][2] = {{xa.x, xa.y}, {xa.z, xa.w}, {xb.x, xb.y}, {xb.z, xb.w}};
+      if (mask & 1u) tile_step(acc[0], rd_codes + so, rd_scales + so, rot, dt, mul_lo, mul_hi, xq, lo, 64u - lo);
+      if (mask & 2u)
+        tile_step(acc[1], rd_codes + so + 128, rd_scales + so + 64, rot, dt, mul_lo, mul_hi, xq, lo, 64u - lo);
+      __syncwarp();                                          // every lane has read the stage: refill it
+      copy_weights(so);
+      copy_x(so);
+      cp_async_commit();
+      cursor_next();
+      so = (so + STAGE_BYTES == DEPTH * STAGE_BYTES) ? 0u : so + STAGE_BYTES;
+    }
+    // End of the unit: leave this warp's partial sums, meet, and let 256 threads finish the rows.
+    // Element (row, token) of the unit sits at row * 8 + token, so a warp's 32 stores hit 32 banks.
+    float* mine = red + (buf * WARPS + warp) * RED_FLOATS;
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         mine[(16 * mt + 8 * (j >> 1) + g) * TOKENS + 2 * t + (j & 1)] = acc[mt][j];
         acc[mt][j] = 0.0f;
       }
     __syncthreads();                                         // the buffer written two units ago was read before the previous meeting
-    if ((int)threadIdx.x < C::RED_FLOATS) {
-      const float* src = red + buf * WARPS * C::RED_FLOATS + threadIdx.x;
+    if ((int)threadIdx.x < RED_FLOATS) {
+      const float* src = red + buf * WARPS * RED_FLOATS + threadIdx.x;
       float s = 0.0f;
 #pragma unroll
-      for (int w = 0; w < WARPS; ++w) s += src[w * C::RED_FLOATS];   // warp order: a fixed summation order
-      const int n = u * C::R + ((int)threadIdx.x >> 3), m = (int)threadIdx.x & 7;
-      if (m < a.M && n < a.g.N) a.y[(size_t)m * a.g.N + n] = __float2bfloat16_rn(ts * s);
+      for (int w = 0; w < WARPS; ++w) s += src[w * RED_FLOATS];      // warp order: a fixed summation order
+      const int row = (int)threadIdx.x >> 3, m = (int)threadIdx.x & 7;
+      const int n = u * UNIT_ROWS + row;
+      if (((mask >> (row >> 4)) & 1u) && m < a.M && n < a.g.N) a.y[(size_t)m * a.g.N + n] = __float2bfloat16_rn(ts * s);
     }
     buf ^= 1;
-  };
-
-  // ---------------- main loop: consume the oldest register set, refill it DEPTH chunks ahead ----------------
-  int cu = u_begin, cc = warp;                               // compute cursor
-  while (cu < u_end) {
-#pragma unroll
-    for (int d = 0; d < DEPTH; ++d) {
-      if (cu < u_end) {
-        compute(regs[d]);
-        if (pu < u_end) {
-          load_w(regs[d], pu, pc);
-          load_x(regs[d], pc);
-        }
-        advance(pu, pc);
-        const int u_done = cu;
-        advance(cu, cc);
-        if (cu != u_done) unit_end(u_done);
-      }
-    }
   }
+  cp_async_wait<0>();
 }
 
 }  // namespace direct_path
@@ -251,24 +292,27 @@ static int direct_sm_count() {
 }
 
 struct DirectPlan {
-  int mt, units, grid;
+  int halves, grid, unit_aligned;
   double balance;            // useful share of the SMs' time: rows are not split over K
 };
 
 static DirectPlan direct_plan(const razer_desc* d) {
   const Geometry g = make_geometry(d->N, d->K);
   const int sms = direct_sm_count();
-  DirectPlan best = {};
-  for (int mt = 2; mt >= 1; --mt) {
-    DirectPlan p;
-    p.mt = mt;
-    p.units = (g.row_tiles * TILE_ROWS) / (16 * mt);
-    p.grid = p.units < sms ? p.units : sms;
-    const int per_cta = (p.units + p.grid - 1) / p.grid;
-    p.balance = (double)p.units / ((double)per_cta * sms);
-    if (mt == 2 || p.balance > best.balance + 0.20) best = p;   // wider units amortise the activation loads
+  DirectPlan p;
+  p.halves = (g.row_tiles * TILE_ROWS) / 16;
+  const int units = (p.halves + 1) / 2;
+  if (units <= sms) {          // one whole 32-row unit per CTA: no unit is walked twice
+    p.grid = units;
+    p.unit_aligned = 1;
+    p.balance = (double)p.halves / (2.0 * sms);
+    return p;
   }
-  return best;
+  p.grid = sms;
+  p.unit_aligned = 0;
+  const int per_cta = (p.halves + p.grid - 1) / p.grid;
+  p.balance = (double)p.halves / ((double)per_cta * sms);
+  return p;
 }
 
 bool gemv_direct_supported(const razer_desc* d, int M) {
@@ -279,13 +323,12 @@ bool gemv_direct_supported(const razer_desc* d, int M) {
 
 double gemv_direct_balance(const razer_desc* d) { return direct_plan(d).balance; }
 
-template <int MT, int DEPTH>
 static int launch_direct_cfg(const direct_path::Args& a, int grid, cudaStream_t st) {
-  using C = direct_path::Cfg<MT>;
-  auto kern = direct_path::razer_direct_kernel<MT, DEPTH>;
+  auto kern = direct_path::razer_direct_kernel;
   static bool attr_set = false;
   if (!attr_set) {
-    RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES),
+    RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)direct_path::SMEM_BYTES),
                          "cudaFuncSetAttribute(max dynamic shared memory)"));
     attr_set = true;
   }
@@ -293,7 +336,7 @@ static int launch_direct_cfg(const direct_path::Args& a, int grid, cudaStream_t 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(direct_path::THREADS);
-  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.dynamicSmemBytes = direct_path::SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -320,9 +363,9 @@ int launch_gemv_direct(const razer_desc* d, const void* packed, const void* x, i
   a.mul_lo = (1u << 6) + (1u << 12);
   a.mul_hi = (1u << 2) + (1u << 8);
   a.M = M;
-  a.units = p.units;
-  if (p.mt == 2) return launch_direct_cfg<2, direct_path::DEPTH_MT2>(a, p.grid, st);
-  return launch_direct_cfg<1, direct_path::DEPTH_MT1>(a, p.grid, st);
+  a.halves = p.halves;
+  a.unit_aligned = p.unit_aligned;
+  return launch_direct_cfg(a, p.grid, st);
 }
 
 }  // namespace razer

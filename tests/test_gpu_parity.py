@@ -260,7 +260,7 @@ import sys, numpy as np, torch
 sys.path.insert(0, sys.argv[1])
 from oracle import razer_oracle as ro
 from paper_2501_04052_b200 import binding as b, inputs
-for (M, N, K, seed) in [(1, 1000, 4160, 1), (5, 333, 2064, 2), (16, 640, 1024, 3), (8, 384, 8192, 4)]:
+for (M, N, K, seed) in [(1, 1000, 4160, 1), (5, 333, 2064, 2), (16, 640, 1024, 3), (8, 384, 8192, 4), (2, 6000, 1088, 5)]:
     codes, scales = inputs.random_codes(N, K, seed=seed, scale_lo=0, scale_hi=64, zero_block_frac=0.02)
     codes, scales = codes.numpy(), scales.numpy()
     desc = b.make_desc(N, K, 0.004, sv_mag=(5.0, 9.0))
@@ -276,10 +276,11 @@ print("ok")
 """
 
 
-@pytest.mark.parametrize("kernel", ["mma", "direct", "simt"])
+@pytest.mark.parametrize("kernel", ["umma", "direct", "mma", "simt"])
 def test_alternative_kernels_match_the_oracle(kernel):
-    """RAZER_KERNEL selects the register-fragment mma.sync kernel or the CUDA-core kernel for the same
-    entry point; the choice is read once per process, so the check runs in a child process."""
+    """RAZER_KERNEL pins the matmul entry points to one kernel (the tcgen05 kernel, the register-only GEMV
+    kernel wherever it can run, the ring-fed mma.sync kernel, or the CUDA-core kernel) instead of the
+    per-shape choice; it is read once per process, so the check runs in a child process."""
     import os
     import subprocess
     import sys
