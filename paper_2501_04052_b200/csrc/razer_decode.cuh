@@ -46,13 +46,16 @@ struct DecodeTables {         // 32-bit shared-window addresses
 
 // Fill the tables (all threads of the CTA call this; a __syncthreads() must follow).
 __device__ __forceinline__ void decode_tables_fill(uint8_t* base, float sv0, float sv1, int tid, int nthreads) {
-  uint32_t* ss = reinterpret_cast<uint32_t*>(base);
-  for (int i = tid; i < DECODE_SS_ENTRIES * 32; i += nthreads) {
-    const uint32_t idx = (uint32_t)i >> 5;
+  // every entry is computed once per quarter (four threads per entry) and written as eight of its 32 lane copies
+  for (int i = tid; i < DECODE_SS_ENTRIES * 4; i += nthreads) {
+    const uint32_t idx = (uint32_t)i >> 2;
     // scale x 2^126 has four significant bits: the upper half of the FP32 pattern is the exact bf16
     const float sc = scale_value(idx & 0x3Fu) * 8.50705917e37f;   // 2^126
     const uint32_t b = (__float_as_uint(sc) >> 16) | ((idx & 0x40u) << 9);
-    ss[i] = b | (b << 16);
+    const uint32_t v = b | (b << 16);
+    uint4* dst = reinterpret_cast<uint4*>(base + idx * 128 + (i & 3) * 32);
+    dst[0] = make_uint4(v, v, v, v);
+    dst[1] = make_uint4(v, v, v, v);
   }
   if (tid < 2) {
     const float sv = tid ? sv1 : sv0;                          // at most four significant bits
