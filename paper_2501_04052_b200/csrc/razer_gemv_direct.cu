@@ -1,23 +1,25 @@
-// Decode GEMV (M <= 8) against packed RaZeR weights for sm_100a: register-only weight path, no split-K
-// through global memory.
+// Decode GEMV (M <= 8) against packed RaZeR weights for sm_100a: register-fragment tensor-core kernel with
+// no exchange between CTAs.
 //
 //   y[m, n] = bf16( ts * sum_k x[m, k] * D1[n, k] ),   D1 = block_scale * element (exact bf16)
 //
-// Every weight byte is used exactly once, so this kernel does not stage weights anywhere: each
-// lane loads the 8-byte code words of "its" blocks straight from global memory into registers
-// (streaming loads, several chunks ahead), decodes them there (razer_decode.cuh) and feeds them
-// as the A fragment of a warp-level m16n8k16 tensor-core MMA whose B fragment is the activation
-// slice (tokens along n), accumulated in FP32 registers.  Sec. 4.3 of the paper describes this style
-// for its weight-only kernel (weights pre-shuffled so that each thread's loads match its MMA fragment).
+// Every weight byte is used exactly once.  Each warp streams "its" chunk slices through a small private
+// ring in shared memory (cp.async, 16 bytes per lane, several slices ahead; only the warp itself waits on
+// them), each lane decodes the code words of "its" blocks in registers (razer_decode.cuh) and feeds them
+// as the A fragment of a warp-level m16n8k16 tensor-core MMA whose B fragment is the activation slice
+// (tokens along n), accumulated in FP32 registers.  Sec. 4.3 of the paper describes this style for its
+// weight-only kernel (weights pre-shuffled so that each thread's loads match its MMA fragment).
 //
-// Work unit: R = 16 * MT weight rows over the whole of K.  A CTA (16 warps) takes a contiguous range of
-// units; inside a unit warp w takes the chunks (64 columns) w, w + 16, ...  In a chunk, lane
-// (g = lane / 4, t = lane % 4) decodes block t of rows g and g + 8 of each 16-row MMA tile; MMA q (0..3)
-// takes elements 4q .. 4q + 3 of every lane's block, i.e. the MMA's k slots are columns
-// 16 t + 4 q + {0, 1, 2, 3}, for A and B alike.  At the end of a unit the 16 warps leave their partial sums
-// in shared memory, and R * 8 threads add them in warp order, scale, round and store.  Nothing is exchanged
-// between CTAs, so there is no workspace, no counter and no wait on another CTA; the price is that the
-// rows have to divide evenly enough over the SMs, which the host checks before it picks this kernel.
+// Work unit: 32 weight rows (two 16-row MMA tiles) over the whole of K.  A CTA (16 warps) takes a contiguous
+// range of rows: whole units when there are no more units than SMs, else 16-row halves (a unit at either end
+// of the range may then be shared with the neighbouring CTA, each doing its own tile).  Inside a unit warp w
+// takes the chunks (64 columns) w, w + 16, ...  In a chunk, lane (g = lane / 4, t = lane % 4) decodes block t
+// of rows g and g + 8 of each tile; MMA q (0..3) takes elements 4q .. 4q + 3 of every lane's block, i.e. the
+// MMA's k slots are columns 16 t + 4 q + {0, 1, 2, 3}, for A and B alike.  At the end of a unit the 16 warps
+// leave their partial sums in shared memory, and 256 threads add them in warp order, scale, round and store.
+// Nothing is exchanged between CTAs, so there is no workspace, no counter and no wait on another CTA; the
+// price is that the rows have to divide evenly enough over the SMs, which the host checks before it picks
+// this kernel.
 #include <cuda.h>
 #include <cstdlib>
 
