@@ -34,7 +34,7 @@ constexpr int WARPS = 16;
 constexpr int THREADS = 32 * WARPS;
 constexpr int TOKENS = 8;
 constexpr int UNIT_ROWS = 32;                       // two 16-row MMA tiles
-constexpr int DEPTH = 4;                            // chunk slices in flight per warp
+constexpr int DEPTH = 2;                            // chunk slices in flight per warp
 // A warp's ring stage: the 32-row slice of one chunk, [blk 0..3][32 slots x 8 B] (blocks 2 and 3 sit 32 bytes
 // further so that a half-warp's 8-byte reads, four blocks x four slots, cover all 32 banks), then
 // [32 rows x 4 scale bytes], then the activations of the chunk: lane l keeps its 16 columns (token l / 4,
