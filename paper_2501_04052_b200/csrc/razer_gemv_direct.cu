@@ -52,12 +52,39 @@ constexpr long long STEP_BYTES = (long long)WARPS * CHUNK_BYTES;   // a warp's n
 
 __device__ __forceinline__ constexpr int stage_blk_off(int blk) { return blk * 256 + (blk >> 1) * 32; }
 
-// 16 bytes, of which only the first `bytes` (0 or 16) are read; the rest is written as zero
+// 16 bytes to dst + DOFF from src + SOFF, of which only the first `bytes` (0 or 16) are read; the rest is written
+// as zero.  The offsets are immediates of the instruction, so one base register serves several copies.
+template <int DOFF, int SOFF>
 __device__ __forceinline__ void cp_async16_cg(uint32_t dst, const void* src, uint32_t bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.cg.shared.global [%0+%3], [%1+%4], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes), "n"(DOFF), "n"(SOFF)
+               : "memory");
 }
+template <int DOFF, int SOFF>
 __device__ __forceinline__ void cp_async16_ca(uint32_t dst, const void* src, uint32_t bytes) {   // kept in L1: re-read per unit
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.ca.shared.global [%0+%3], [%1+%4], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes), "n"(DOFF), "n"(SOFF)
+               : "memory");
+}
+// shared-memory loads at base + OFF (immediate)
+template <int OFF>
+__device__ __forceinline__ uint32_t lds32_at(uint32_t base) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(base), "n"(OFF) : "memory");
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint2 lds64_at(uint32_t base) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(base), "n"(OFF) : "memory");
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint4 lds128_at(uint32_t base) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4+%5];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "r"(base), "n"(OFF)
+               : "memory");
+  return v;
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -85,13 +112,15 @@ struct Args {
   int unit_aligned;          // every CTA owns whole 32-row units (grid = units)
 };
 
-// One chunk slice of one MMA tile (16 rows): decode the lane's two blocks, four MMAs.
-// rot = (8 t + 25) % 32 turns the row's scale word so that block t's byte sits on bits 14:7.
-__device__ __forceinline__ void tile_step(float (&acc)[4], uint32_t st_codes, uint32_t st_scales, uint32_t rot,
-                                          const DecodeTables& dt, uint32_t mul_lo, uint32_t mul_hi,
-                                          const uint32_t (&xq)[4][2], uint32_t off_h0, uint32_t off_h1) {
-  const uint2 c0 = lds64(st_codes + off_h0), c1 = lds64(st_codes + off_h1);
-  const uint32_t s0 = lds32(st_scales), s1 = lds32(st_scales + 32);
+// One chunk slice of MMA tile TILE (16 rows): decode the lane's two blocks, four MMAs.
+// codes_h0 / codes_h1: the lane's code words of rows g / g + 8 of tile 0 in the stage; scales: row g's scale word.
+// rot = (8 t + 25) % 32 turns a row's scale word so that block t's byte sits on bits 14:7.
+template <int TILE>
+__device__ __forceinline__ void tile_step(float (&acc)[4], uint32_t codes_h0, uint32_t codes_h1, uint32_t scales,
+                                          uint32_t rot, const DecodeTables& dt, uint32_t mul_lo, uint32_t mul_hi,
+                                          const uint32_t (&xq)[4][2]) {
+  const uint2 c0 = lds64_at<128 * TILE>(codes_h0), c1 = lds64_at<128 * TILE>(codes_h1);
+  const uint32_t s0 = lds32_at<64 * TILE>(scales), s1 = lds32_at<64 * TILE + 32>(scales);
   uint32_t e[2][8];
   {
     uint32_t ss2;
@@ -143,6 +172,7 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
 
   const uint32_t ring = smem_addr(ring_base) + (uint32_t)warp * (DEPTH * STAGE_BYTES);
   const bool has_token = g < a.M;
+  const bool k_tail = (a.g.K % CHUNK_K) != 0;                // only then can a chunk hold absent columns
   // ---- copy side: what this lane copies for every chunk slice ----
   // two 16-byte pieces of code words (blocks cblk and cblk + 2, slots 2 piece and + 1), 16 bytes of scale
   // words (lanes 0..7) and its own 32 bytes of activations; a size of 0 writes zeros and reads nothing
@@ -169,17 +199,22 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   };
   auto copy_weights = [&](uint32_t so) {                     // weights: no dependency on earlier kernels
     if (cp_unit < u_end) {
-      cp_async16_cg(dst_codes + so, src_codes, sz_codes);
-      cp_async16_cg(dst_codes + so + 544, src_codes + 2048, sz_codes);
-      if (lane < 8) cp_async16_cg(dst_lane + so + STAGE_CODE_BYTES, src_scales, sz_scales);
+      const uint32_t dc = dst_codes + so;
+      cp_async16_cg<0, 0>(dc, src_codes, sz_codes);
+      cp_async16_cg<544, 2048>(dc, src_codes, sz_codes);
+      if (lane < 8) cp_async16_cg<STAGE_CODE_BYTES, 0>(dst_lane + so, src_scales, sz_scales);
     }
   };
   auto copy_x = [&](uint32_t so) {
     if (has_token && cp_unit < u_end) {
-      const bool in = col < a.g.K;                           // K is a multiple of 16: a 16-column group is whole
-      const __nv_bfloat16* src = in ? src_x : a.x;
-      cp_async16_ca(dst_lane + so + STAGE_X_OFF, src, in ? 16u : 0u);
-      cp_async16_ca(dst_lane + so + STAGE_X_OFF + 512, src + 8, in ? 16u : 0u);
+      const __nv_bfloat16* src = src_x;
+      uint32_t sz = 16u;
+      if (k_tail && col >= a.g.K) {                          // K is a multiple of 16: a 16-column group is whole or absent
+        src = a.x;
+        sz = 0u;
+      }
+      cp_async16_ca<STAGE_X_OFF, 0>(dst_lane + so, src, sz);
+      cp_async16_ca<STAGE_X_OFF + 512, 16>(dst_lane + so, src, sz);
     }
   };
   auto cursor_next = [&]() {
@@ -226,7 +261,7 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
 
   // ---- compute side: this lane's reads from a stage ----
   const uint32_t lo = (t & 1) ? 64u : 0u;                    // odd blocks keep rows g and g + 8 the other way round
-  const uint32_t rd_codes = ring + stage_blk_off(t) + g * 8;
+  const uint32_t rd_h0 = ring + stage_blk_off(t) + g * 8 + lo, rd_h1 = ring + stage_blk_off(t) + g * 8 + (64u - lo);
   const uint32_t rd_scales = ring + STAGE_CODE_BYTES + g * 4;
   const uint32_t rot = (uint32_t)(8 * t + 25) & 31u;
   float acc[2][4];
@@ -243,17 +278,18 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
     for (int j = 0; j < per_unit; ++j) {
       cp_async_wait<DEPTH - 1>();                            // this lane's pieces of the oldest slice have landed
       __syncwarp();                                          // ... and so have the other lanes'
-      const uint4 xa = lds128(dst_lane + so + STAGE_X_OFF), xb = lds128(dst_lane + so + STAGE_X_OFF + 512);
+      const uint32_t bx = dst_lane + so, bh0 = rd_h0 + so, bh1 = rd_h1 + so, bs = rd_scales + so;
+      const uint4 xa = lds128_at<STAGE_X_OFF>(bx), xb = lds128_at<STAGE_X_OFF + 512>(bx);
       const uint32_t xq[4][2] = {{xa.x, xa.y}, {xa.z, xa.w}, {xb.x, xb.y}, {xb.z, xb.w}};
-      if (mask & 1u) tile_step(acc[0], rd_codes + so, rd_scales + so, rot, dt, mul_lo, mul_hi, xq, lo, 64u - lo);
-      if (mask & 2u)
-        tile_step(acc[1], rd_codes + so + 128, rd_scales + so + 64, rot, dt, mul_lo, mul_hi, xq, lo, 64u - lo);
+      if (mask & 1u) tile_step<0>(acc[0], bh0, bh1, bs, rot, dt, mul_lo, mul_hi, xq);
+      if (mask & 2u) tile_step<1>(acc[1], bh0, bh1, bs, rot, dt, mul_lo, mul_hi, xq);
       __syncwarp();                                          // every lane has read the stage: refill it
       copy_weights(so);
       copy_x(so);
       cp_async_commit();
       cursor_next();
-      so = (so + STAGE_BYTES == DEPTH * STAGE_BYTES) ? 0u : so + STAGE_BYTES;
+      if (DEPTH == 2) so ^= (uint32_t)STAGE_BYTES;
+      else so = (so + STAGE_BYTES == DEPTH * STAGE_BYTES) ? 0u : so + STAGE_BYTES;
     }
     // End of the unit: leave this warp's partial sums, meet, and let 256 threads finish the rows.
     // Element (row, token) of the unit sits at row * 8 + token, so a warp's 32 stores hit 32 banks.
