@@ -1,4 +1,4 @@
-// Decode GEMV (M <= 8) against packed RaZeR weights for sm_100a: register-fragment tensor-core kernel with
+// Decode GEMV (M <= 16) against packed RaZeR weights for sm_100a: register-fragment tensor-core kernel with
 // no exchange between CTAs.
 //
 //   y[m, n] = bf16( ts * sum_k x[m, k] * D1[n, k] ),   D1 = block_scale * element (exact bf16)
@@ -7,7 +7,7 @@
 // ring in shared memory (cp.async, 16 bytes per lane, several slices ahead; only the warp itself waits on
 // them), each lane decodes the code words of "its" blocks in registers (razer_decode.cuh) and feeds them
 // as the A fragment of a warp-level m16n8k16 tensor-core MMA whose B fragment is the activation slice
-// (tokens along n), accumulated in FP32 registers.  Sec. 4.3 of the paper describes this style for its
+// (8 tokens along n; a second fragment and accumulator for tokens 8..15), accumulated in FP32 registers.  Sec. 4.3 of the paper describes this style for its
 // weight-only kernel (weights pre-shuffled so that each thread's loads match its MMA fragment).
 //
 // Work unit: 32 weight rows (two 16-row MMA tiles) over the whole of K.  A CTA (16 warps) takes a contiguous
@@ -16,7 +16,7 @@
 // takes the chunks (64 columns) w, w + 16, ...  In a chunk, lane (g = lane / 4, t = lane % 4) decodes block t
 // of rows g and g + 8 of each tile; MMA q (0..3) takes elements 4q .. 4q + 3 of every lane's block, i.e. the
 // MMA's k slots are columns 16 t + 4 q + {0, 1, 2, 3}, for A and B alike.  At the end of a unit the 16 warps
-// leave their partial sums in shared memory, and 256 threads add them in warp order, scale, round and store.
+// leave their partial sums in shared memory, and 32 x tokens threads add them in warp order, scale, round and store.
 // Nothing is exchanged between CTAs, so there is no workspace, no counter and no wait on another CTA; the
 // price is that the rows have to divide evenly enough over the SMs, which the host checks before it picks
 // this kernel.
@@ -32,23 +32,28 @@ namespace direct_path {
 
 constexpr int WARPS = 16;
 constexpr int THREADS = 32 * WARPS;
-constexpr int TOKENS = 8;
 constexpr int UNIT_ROWS = 32;                       // two 16-row MMA tiles
 constexpr int DEPTH = 2;                            // chunk slices in flight per warp
 // A warp's ring stage: the 32-row slice of one chunk, [blk 0..3][32 slots x 8 B] (blocks 2 and 3 sit 32 bytes
 // further so that a half-warp's 8-byte reads, four blocks x four slots, cover all 32 banks), then
-// [32 rows x 4 scale bytes], then the activations of the chunk: lane l keeps its 16 columns (token l / 4,
-// columns 16 (l % 4) ..) as two 16-byte halves at 16 l and 512 + 16 l.
+// [32 rows x 4 scale bytes], then per group of 8 tokens the activations of the chunk: lane l keeps its 16 columns
+// (token l / 4 of the group, columns 16 (l % 4) ..) as two 16-byte halves at 16 l and 512 + 16 l.
 constexpr int STAGE_CODE_BYTES = 4 * 256 + 32;
 constexpr int STAGE_X_OFF = STAGE_CODE_BYTES + 128;
-constexpr int STAGE_BYTES = STAGE_X_OFF + 1024;
-constexpr int RED_FLOATS = UNIT_ROWS * TOKENS;      // one warp's partial sums
-constexpr int RED_BYTES = 2 * WARPS * RED_FLOATS * 4;
-constexpr int RING_BYTES = WARPS * DEPTH * STAGE_BYTES;
 constexpr int TABLE_ALIGN = 16384;                  // decode_block_consts_rot() wants the tables on a 16 KB boundary
-constexpr size_t SMEM_BYTES = TABLE_ALIGN + DECODE_TABLE_BYTES + RING_BYTES + RED_BYTES;
-static_assert(STAGE_BYTES % 16 == 0 && STAGE_X_OFF % 16 == 0 && DECODE_TABLE_BYTES % 16 == 0, "16-byte copies");
 constexpr long long STEP_BYTES = (long long)WARPS * CHUNK_BYTES;   // a warp's next chunk of the same unit
+static_assert(STAGE_X_OFF % 16 == 0 && DECODE_TABLE_BYTES % 16 == 0, "16-byte copies");
+
+template <int NT>                                   // NT groups of 8 tokens
+struct Cfg {
+  static constexpr int TOKENS = 8 * NT;
+  static constexpr int STAGE_BYTES = STAGE_X_OFF + 1024 * NT;
+  static constexpr int RED_FLOATS = UNIT_ROWS * TOKENS;      // one warp's partial sums
+  static constexpr int RED_BYTES = 2 * WARPS * RED_FLOATS * 4;
+  static constexpr int RING_BYTES = WARPS * DEPTH * STAGE_BYTES;
+  static constexpr size_t SMEM_BYTES = TABLE_ALIGN + DECODE_TABLE_BYTES + RING_BYTES + RED_BYTES;
+  static_assert(RED_FLOATS <= THREADS && SMEM_BYTES <= 227 * 1024, "one thread per output of a unit; one CTA per SM");
+};
 
 __device__ __forceinline__ constexpr int stage_blk_off(int blk) { return blk * 256 + (blk >> 1) * 32; }
 
@@ -115,10 +120,10 @@ struct Args {
 // One chunk slice of MMA tile TILE (16 rows): decode the lane's two blocks, four MMAs.
 // codes_h0 / codes_h1: the lane's code words of rows g / g + 8 of tile 0 in the stage; scales: row g's scale word.
 // rot = (8 t + 25) % 32 turns a row's scale word so that block t's byte sits on bits 14:7.
-template <int TILE>
-__device__ __forceinline__ void tile_step(float (&acc)[4], uint32_t codes_h0, uint32_t codes_h1, uint32_t scales,
+template <int TILE, int NT>
+__device__ __forceinline__ void tile_step(float (&acc)[NT][4], uint32_t codes_h0, uint32_t codes_h1, uint32_t scales,
                                           uint32_t rot, const DecodeTables& dt, uint32_t mul_lo, uint32_t mul_hi,
-                                          const uint32_t (&xq)[4][2]) {
+                                          const uint32_t (&xq)[NT][4][2]) {
   const uint2 c0 = lds64_at<128 * TILE>(codes_h0), c1 = lds64_at<128 * TILE>(codes_h1);
   const uint32_t s0 = lds32_at<64 * TILE>(scales), s1 = lds32_at<64 * TILE + 32>(scales);
   uint32_t e[2][8];
@@ -138,10 +143,15 @@ __device__ __forceinline__ void tile_step(float (&acc)[4], uint32_t codes_h0, ui
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q)
-    mma_16816(acc, e[0][2 * q], e[1][2 * q], e[0][2 * q + 1], e[1][2 * q + 1], xq[q][0], xq[q][1]);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+      mma_16816(acc[nt], e[0][2 * q], e[1][2 * q], e[0][2 * q + 1], e[1][2 * q + 1], xq[nt][q][0], xq[nt][q][1]);
 }
 
+template <int NT>
 __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) {
+  using C = Cfg<NT>;
+  constexpr int TOKENS = C::TOKENS, STAGE_BYTES = C::STAGE_BYTES, RED_FLOATS = C::RED_FLOATS, RING_BYTES = C::RING_BYTES;
   extern __shared__ __align__(16) uint8_t smem_raw[];
   // tables first, on a 16 KB boundary of the shared window; then the rings; then the reduction buffers
   const uint32_t raw_addr = smem_addr(smem_raw);
@@ -171,7 +181,9 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   decode_tables_fill(tables, a.sv0, a.sv1, threadIdx.x, THREADS);
 
   const uint32_t ring = smem_addr(ring_base) + (uint32_t)warp * (DEPTH * STAGE_BYTES);
-  const bool has_token = g < a.M;
+  bool has_token[NT];                                        // token g of group nt exists
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) has_token[nt] = 8 * nt + g < a.M;
   const bool k_tail = (a.g.K % CHUNK_K) != 0;                // only then can a chunk hold absent columns
   // ---- copy side: what this lane copies for every chunk slice ----
   // two 16-byte pieces of code words (blocks cblk and cblk + 2, slots 2 piece and + 1), 16 bytes of scale
@@ -181,7 +193,7 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   const uint32_t dst_lane = ring + lane * 16;                                 // + STAGE_CODE_BYTES: scales, + STAGE_X_OFF: activations
   const uint8_t* src_codes;                                                   // blocks cblk + 2: 2048 bytes further
   const uint8_t* src_scales;
-  const __nv_bfloat16* src_x;
+  const __nv_bfloat16* src_x;                                                 // token g; token g + 8: 8 K elements further
   int col, cp_unit, cp_left;                                                  // first activation column; unit; chunks of it still to copy
   uint32_t sz_codes, sz_scales;
   auto cursor_to_unit = [&](int u) {
@@ -190,7 +202,7 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
     const uint32_t mask = u < u_end ? unit_mask(u) : 0u;
     src_codes = ck + r0 * 8 + cblk * 1024 + piece * 16;
     src_scales = ck + CHUNK_CODE_BYTES + r0 * 4 + (lane & 7) * 16;
-    src_x = a.x + (size_t)(has_token ? g : 0) * a.g.K + warp * CHUNK_K + 16 * t;
+    src_x = a.x + (size_t)(has_token[0] ? g : 0) * a.g.K + warp * CHUNK_K + 16 * t;
     col = warp * CHUNK_K + 16 * t;
     cp_unit = u;
     cp_left = per_unit;
@@ -206,15 +218,25 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
     }
   };
   auto copy_x = [&](uint32_t so) {
-    if (has_token && cp_unit < u_end) {
-      const __nv_bfloat16* src = src_x;
-      uint32_t sz = 16u;
-      if (k_tail && col >= a.g.K) {                          // K is a multiple of 16: a 16-column group is whole or absent
-        src = a.x;
-        sz = 0u;
+    if (cp_unit < u_end) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        if (has_token[nt]) {
+          const __nv_bfloat16* src = src_x + (size_t)nt * 8 * a.g.K;
+          uint32_t sz = 16u;
+          if (k_tail && col >= a.g.K) {                      // K is a multiple of 16: a 16-column group is whole or absent
+            src = a.x;
+            sz = 0u;
+          }
+          if (nt == 0) {
+            cp_async16_ca<STAGE_X_OFF, 0>(dst_lane + so, src, sz);
+            cp_async16_ca<STAGE_X_OFF + 512, 16>(dst_lane + so, src, sz);
+          } else {
+            cp_async16_ca<STAGE_X_OFF + 1024, 0>(dst_lane + so, src, sz);
+            cp_async16_ca<STAGE_X_OFF + 1536, 16>(dst_lane + so, src, sz);
+          }
+        }
       }
-      cp_async16_ca<STAGE_X_OFF, 0>(dst_lane + so, src, sz);
-      cp_async16_ca<STAGE_X_OFF + 512, 16>(dst_lane + so, src, sz);
     }
   };
   auto cursor_next = [&]() {
@@ -229,14 +251,16 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   };
 
   // lanes without a token never copy activations: their slots stay zero
-  if (!has_token) {
-    uint8_t* mine = ring_base + (size_t)warp * (DEPTH * STAGE_BYTES) + STAGE_X_OFF + lane * 16;
 #pragma unroll
-    for (int d = 0; d < DEPTH; ++d) {
-      *reinterpret_cast<uint4*>(mine + d * STAGE_BYTES) = make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4*>(mine + d * STAGE_BYTES + 512) = make_uint4(0, 0, 0, 0);
+  for (int nt = 0; nt < NT; ++nt)
+    if (!has_token[nt]) {
+      uint8_t* mine = ring_base + (size_t)warp * (DEPTH * STAGE_BYTES) + STAGE_X_OFF + 1024 * nt + lane * 16;
+#pragma unroll
+      for (int d = 0; d < DEPTH; ++d) {
+        *reinterpret_cast<uint4*>(mine + d * STAGE_BYTES) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(mine + d * STAGE_BYTES + 512) = make_uint4(0, 0, 0, 0);
+      }
     }
-  }
 
   // ---------------- prologue: the first DEPTH slices' weights, then (after the dependency) their activations ----------------
   cursor_to_unit(u_begin);
@@ -264,11 +288,13 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   const uint32_t rd_h0 = ring + stage_blk_off(t) + g * 8 + lo, rd_h1 = ring + stage_blk_off(t) + g * 8 + (64u - lo);
   const uint32_t rd_scales = ring + STAGE_CODE_BYTES + g * 4;
   const uint32_t rot = (uint32_t)(8 * t + 25) & 31u;
-  float acc[2][4];
+  float acc[2][NT][4];
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[mt][j] = 0.0f;
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[mt][nt][j] = 0.0f;
 
   uint32_t so = 0;                                           // byte offset of the current stage in the ring
   int buf = 0;
@@ -279,10 +305,19 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
       cp_async_wait<DEPTH - 1>();                            // this lane's pieces of the oldest slice have landed
       __syncwarp();                                          // ... and so have the other lanes'
       const uint32_t bx = dst_lane + so, bh0 = rd_h0 + so, bh1 = rd_h1 + so, bs = rd_scales + so;
-      const uint4 xa = lds128_at<STAGE_X_OFF>(bx), xb = lds128_at<STAGE_X_OFF + 512>(bx);
-      const uint32_t xq[4][2] = {{xa.x, xa.y}, {xa.z, xa.w}, {xb.x, xb.y}, {xb.z, xb.w}};
-      if (mask & 1u) tile_step<0>(acc[0], bh0, bh1, bs, rot, dt, mul_lo, mul_hi, xq);
-      if (mask & 2u) tile_step<1>(acc[1], bh0, bh1, bs, rot, dt, mul_lo, mul_hi, xq);
+      uint32_t xq[NT][4][2];
+      {
+        const uint4 xa = lds128_at<STAGE_X_OFF>(bx), xb = lds128_at<STAGE_X_OFF + 512>(bx);
+        xq[0][0][0] = xa.x, xq[0][0][1] = xa.y, xq[0][1][0] = xa.z, xq[0][1][1] = xa.w;
+        xq[0][2][0] = xb.x, xq[0][2][1] = xb.y, xq[0][3][0] = xb.z, xq[0][3][1] = xb.w;
+      }
+      if (NT == 2) {
+        const uint4 xa = lds128_at<STAGE_X_OFF + 1024>(bx), xb = lds128_at<STAGE_X_OFF + 1536>(bx);
+        xq[NT - 1][0][0] = xa.x, xq[NT - 1][0][1] = xa.y, xq[NT - 1][1][0] = xa.z, xq[NT - 1][1][1] = xa.w;
+        xq[NT - 1][2][0] = xb.x, xq[NT - 1][2][1] = xb.y, xq[NT - 1][3][0] = xb.z, xq[NT - 1][3][1] = xb.w;
+      }
+      if (mask & 1u) tile_step<0, NT>(acc[0], bh0, bh1, bs, rot, dt, mul_lo, mul_hi, xq);
+      if (mask & 2u) tile_step<1, NT>(acc[1], bh0, bh1, bs, rot, dt, mul_lo, mul_hi, xq);
       __syncwarp();                                          // every lane has read the stage: refill it
       copy_weights(so);
       copy_x(so);
@@ -292,22 +327,24 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
       else so = (so + STAGE_BYTES == DEPTH * STAGE_BYTES) ? 0u : so + STAGE_BYTES;
     }
     // End of the unit: leave this warp's partial sums, meet, and let 256 threads finish the rows.
-    // Element (row, token) of the unit sits at row * 8 + token, so a warp's 32 stores hit 32 banks.
+    // Element (row, token) of the unit sits at row * TOKENS + token (8 tokens: a warp's 32 stores hit 32 banks).
     float* mine = red + (buf * WARPS + warp) * RED_FLOATS;
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        mine[(16 * mt + 8 * (j >> 1) + g) * TOKENS + 2 * t + (j & 1)] = acc[mt][j];
-        acc[mt][j] = 0.0f;
-      }
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          mine[(16 * mt + 8 * (j >> 1) + g) * TOKENS + 8 * nt + 2 * t + (j & 1)] = acc[mt][nt][j];
+          acc[mt][nt][j] = 0.0f;
+        }
     __syncthreads();                                         // the buffer written two units ago was read before the previous meeting
     if ((int)threadIdx.x < RED_FLOATS) {
       const float* src = red + buf * WARPS * RED_FLOATS + threadIdx.x;
       float s = 0.0f;
 #pragma unroll
       for (int w = 0; w < WARPS; ++w) s += src[w * RED_FLOATS];      // warp order: a fixed summation order
-      const int row = (int)threadIdx.x >> 3, m = (int)threadIdx.x & 7;
+      const int row = (int)threadIdx.x / TOKENS, m = (int)threadIdx.x % TOKENS;
       const int n = u * UNIT_ROWS + row;
       if (((mask >> (row >> 4)) & 1u) && m < a.M && n < a.g.N) a.y[(size_t)m * a.g.N + n] = __float2bfloat16_rn(ts * s);
     }
@@ -355,18 +392,19 @@ static DirectPlan direct_plan(const razer_desc* d) {
 
 bool gemv_direct_supported(const razer_desc* d, int M) {
   const Geometry g = make_geometry(d->N, d->K);
-  return M >= 1 && M <= direct_path::TOKENS && g.k_chunks >= direct_path::WARPS &&
+  return M >= 1 && M <= 16 && g.k_chunks >= direct_path::WARPS &&
          (long long)g.row_tiles * g.k_chunks < (1ll << 30);
 }
 
 double gemv_direct_balance(const razer_desc* d) { return direct_plan(d).balance; }
 
+template <int NT>
 static int launch_direct_cfg(const direct_path::Args& a, int grid, cudaStream_t st) {
-  auto kern = direct_path::razer_direct_kernel;
+  using C = direct_path::Cfg<NT>;
+  auto kern = direct_path::razer_direct_kernel<NT>;
   static bool attr_set = false;
   if (!attr_set) {
-    RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)direct_path::SMEM_BYTES),
+    RAZER_TRY(check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES),
                          "cudaFuncSetAttribute(max dynamic shared memory)"));
     attr_set = true;
   }
@@ -374,7 +412,7 @@ static int launch_direct_cfg(const direct_path::Args& a, int grid, cudaStream_t 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(direct_path::THREADS);
-  cfg.dynamicSmemBytes = direct_path::SMEM_BYTES;
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -403,7 +441,7 @@ int launch_gemv_direct(const razer_desc* d, const void* packed, const void* x, i
   a.M = M;
   a.halves = p.halves;
   a.unit_aligned = p.unit_aligned;
-  return launch_direct_cfg(a, p.grid, st);
+  return M <= 8 ? launch_direct_cfg<1>(a, p.grid, st) : launch_direct_cfg<2>(a, p.grid, st);
 }
 
 }  // namespace razer
