@@ -123,8 +123,11 @@ int razer_gemm(const razer_desc* d, const void* packed_dev, const void* x_dev, i
                void* y_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 
 /* razer_gemv with HOST activations and HOST output: copies x (M*K bf16) into
- * x_stage_dev, runs razer_gemv, copies y (M*N bf16) back and synchronizes the stream.
- * x_host / y_host should be pinned for the copies to be asynchronous. */
+ * x_stage_dev, runs razer_gemv, brings y (M*N bf16) back and synchronizes the stream.
+ * x_host / y_host should be pinned for the copies to be asynchronous.  When y_host is
+ * pinned memory that the device can address (what cudaHostAlloc / cudaHostRegister give
+ * under unified addressing), the kernel stores y straight into it and y_stage_dev is not
+ * touched; otherwise y goes through y_stage_dev and one more copy. */
 int razer_gemv_host(const razer_desc* d, const void* packed_dev, const void* x_host, int M,
                     void* y_host, void* x_stage_dev, void* y_stage_dev, void* workspace_dev,
                     size_t workspace_bytes, void* stream);

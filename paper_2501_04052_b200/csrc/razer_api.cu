@@ -240,13 +240,25 @@ int razer_gemv_host(const razer_desc* d, const void* packed_dev, const void* x_h
   RAZER_TRY(check_ptr(x_stage_dev, 16, "x_stage_dev"));
   RAZER_TRY(check_ptr(y_stage_dev, 2, "y_stage_dev"));
   cudaStream_t st = (cudaStream_t)stream;
+  // pinned host memory that the device can address takes the kernel's stores directly (no copy back)
+  void* y_target = y_stage_dev;
+  {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, y_host) == cudaSuccess) {
+      if (at.type == cudaMemoryTypeHost && at.devicePointer) y_target = at.devicePointer;
+    } else {
+      cudaGetLastError();                                    // not a CUDA-known pointer: use the staging buffer
+    }
+  }
   RAZER_TRY(check_cuda(cudaMemcpyAsync(x_stage_dev, x_host, (size_t)M * d->K * 2, cudaMemcpyHostToDevice, st),
                        "copy of x to the device"));
-  RAZER_TRY(matmul_common(d, packed_dev, x_stage_dev, M, y_stage_dev, workspace_dev, workspace_bytes, 1.0f,
+  RAZER_TRY(matmul_common(d, packed_dev, x_stage_dev, M, y_target, workspace_dev, workspace_bytes, 1.0f,
                           nullptr, st));
-  RAZER_TRY(check_cuda(cudaMemcpyAsync(y_host, y_stage_dev, (size_t)M * d->N * 2, cudaMemcpyDeviceToHost, st),
-                       "copy of y to the host"));
-  if (workspace_dev) return razer_workspace_status(workspace_dev, stream);   // synchronizes
+  if (y_target == y_stage_dev)
+    RAZER_TRY(check_cuda(cudaMemcpyAsync(y_host, y_stage_dev, (size_t)M * d->N * 2, cudaMemcpyDeviceToHost, st),
+                         "copy of y to the host"));
+  // the register-fragment kernel has no device-side wait that could give up: nothing to read back for it
+  if (workspace_dev && !use_direct(d, M)) return razer_workspace_status(workspace_dev, stream);   // synchronizes
   return check_cuda(cudaStreamSynchronize(st), "stream synchronize");
 }
 

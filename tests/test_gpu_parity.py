@@ -226,18 +226,25 @@ def test_w4a4_config5_full_size_sampled_rows(b):
 
 # ------------------------------------------------------------------ host-buffer entry point, errors
 
-def test_gemv_host_entry_point(b):
-    N, K, M = 512, 1024, 2
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("M,N,K", [(2, 512, 1024), (40, 300, 528)])
+def test_gemv_host_entry_point(b, pinned, M, N, K):
+    """Host x in, host y out.  Pinned y takes the kernel's stores directly, pageable y goes through the staging
+    buffer; (2, 512, 1024) runs on the register-fragment kernel, (40, 300, 528) on the tcgen05 kernel."""
     codes, scales = inputs.random_codes(N, K, seed=97)
     desc, packed = _pack(b, codes.numpy(), scales.numpy(), 0.01)
-    x = inputs.activations(M, K, 97).pin_memory()
-    y = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    x = inputs.activations(M, K, 97)
+    y = torch.full((M, N), float("nan"), dtype=torch.bfloat16)
+    if pinned:
+        x, y = x.pin_memory(), y.pin_memory()
     xs = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
     ys = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     ws = b.alloc_workspace(desc, M, b.OP_GEMV, "cuda")
-    b.razer_gemv_host(desc, packed, x, y, xs, ys, ws)
-    y_dev = b.razer_gemv(desc, packed, x.cuda())
-    assert torch.equal(y, y_dev.cpu())
+    for _ in range(2):
+        b.razer_gemv_host(desc, packed, x, y, xs, ys, ws)
+        y_dev = b.razer_gemv(desc, packed, x.cuda())
+        assert torch.equal(y, y_dev.cpu())
+        y.fill_(float("nan"))
 
 
 def test_workspace_too_small_is_an_error(b):
