@@ -332,7 +332,7 @@ def main():
         y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
         ws = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
         ac, as_, ats = b.razer_quant_act(x)
-        tq = time_cuda(lambda i: b.razer_quant_act(x), 20, torch)
+        tq = graph_time(lambda i: b.razer_quant_act(x), 8)
         f = lambda i: b.razer_gemm_w4a4(desc, sets[i % 4], ac, as_, ats, y=y, workspace=ws)
         for i in range(3):
             f(i)
