@@ -33,6 +33,9 @@ if ROOT not in sys.path:
 DECODE_SHAPES = [(4096, 4096), (11008, 4096), (4096, 11008)]
 SKINNY_SHAPES = [(8192, 8192), (28672, 8192), (8192, 28672)]
 PREFILL_SHAPES = [(14336, 4096), (4096, 14336)]
+# DRAM bytes of one step (its three launches) read from the ncu capture of the kernel as committed:
+# 9,464,320 + 25,389,568 + 25,403,392 read, 0 written.  Set to None whenever the kernel changes until re-captured.
+NCU_DRAM_BYTES_PER_STEP = 60257280
 METRIC = "razer_gemv_effective_hbm_bandwidth"
 
 
@@ -285,7 +288,9 @@ def main():
         "timing": "CUDA events around one replay of a CUDA graph holding the K steps",
         "stream_launch": {"value": world * step_bytes / (ms_stream * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms_stream},
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": pk["hbm"], "unit": "GB/s",
-                     "frac": value / world / pk["hbm"], "traffic": None, "peak_source": pk["source"],
+                     "frac": value / world / pk["hbm"], "traffic": NCU_DRAM_BYTES_PER_STEP, "peak_source": pk["source"],
+                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the step's three launches "
+                                       "(profiles/razer_direct_kernel_gemv_config2.md)",
                      "kernel": "razer_gemv (3 launches per step)", "algorithmic_bytes_per_step": step_bytes,
                      "frac_of_nominal_8TBps": value / world / 8000.0},
         "decode_per_shape": per_shape,

@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
       else so = (so + STAGE_BYTES == DEPTH * STAGE_BYTES) ? 0u : so + STAGE_BYTES;
     }
     // End of the unit: leave this warp's partial sums, meet, and let 256 threads finish the rows.
-    // Element (row, token) of the unit sits at row * TOKENS + token (8 tokens: a warp's 32 stores hit 32 banks).
+    // Element (row, token) of the unit sits at row * TOKENS + token (8 tokens: a warp's 32 stores fall on 16 banks, two each; 8 stores per unit).
     float* mine = red + (buf * WARPS + warp) * RED_FLOATS;
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
