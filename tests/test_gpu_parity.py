@@ -194,7 +194,7 @@ def test_quant_act_given_scale_and_zero_input(b):
     assert ts.item() == 1.0 and not codes.any() and not scales.any()
 
 
-@pytest.mark.parametrize("M,N,K", [(256, 1024, 8192), (17, 200, 464)])
+@pytest.mark.parametrize("M,N,K", [(256, 1024, 8192), (17, 200, 464), (8, 300, 2048), (13, 520, 1040)])
 def test_w4a4_oracle_quantized(b, M, N, K):
     """BASELINE config 5 (rows of N sampled down to keep the oracle quantizer quick)."""
     w, wc, ws, wd = oracle_quantized_weights(N, K, 4)
