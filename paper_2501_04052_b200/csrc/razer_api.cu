@@ -84,8 +84,8 @@ double gemv_direct_balance(const razer_desc*);
 
 // Kernel choice.  The tcgen05 kernel serves every M.  For M <= 16 the register-fragment kernel without split-K
 // (razer_gemv_direct.cu) is faster whenever its fixed cost matters or the rows divide well over the SMs
-// (measured on B200: 5.8 against 12.7 us for 4096 x 4096, level at 132 MB with 28672 rows, behind at 132 MB with
-// 8192 rows), so it takes those shapes; with 9 to 16 tokens only the small ones.  RAZER_KERNEL (environment, read once) overrides: "umma" keeps
+// (measured on B200: 5.1 against 12.7 us for 4096 x 4096, 47.7 against 50.0 at 8192 x 28672, level at 6144 x 28672,
+// 39.8 against 35.3 at 5120 x 28672 where its busiest CTA does 1.5 times the average), so it takes those shapes; with 9 to 16 tokens only the small ones.  RAZER_KERNEL (environment, read once) overrides: "umma" keeps
 // everything on the tcgen05 kernel, "direct" takes the register kernel wherever it is able to run, "mma"
 // routes M <= 16 to the older ring-fed mma.sync kernel (kept for comparison), "simt" routes everything to
 // the CUDA-core kernel (debugging aid).
@@ -103,7 +103,7 @@ static bool use_direct(const razer_desc* d, int M) {
   // 9..16 tokens: a 32-row unit re-reads 1.8 times its own weight bytes of activations from L2, so only while
   // the launch's fixed cost dominates (measured: 7.1 against 13.0 us at 4096 x 4096, 26.0 against 20.7 at 8192 x 8192)
   if (M > 8) return bytes <= ((size_t)28 << 20);
-  return bytes <= ((size_t)64 << 20) || gemv_direct_balance(d) >= 0.9;
+  return bytes <= ((size_t)64 << 20) || gemv_direct_balance(d) >= 0.8;
 }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

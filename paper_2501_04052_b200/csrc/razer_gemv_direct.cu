@@ -114,7 +114,7 @@ struct Args {
   float sv0, sv1, tensor_scale;
   uint32_t mul_lo, mul_hi;   // 2^6 + 2^12 and 2^2 + 2^8 (razer_decode.cuh)
   int M, halves;             // 16-row half units of the padded matrix
-  int unit_aligned;          // every CTA owns whole 32-row units (grid = units)
+  int unit_aligned;          // CTA ranges are whole 32-row units (else 16-row halves)
 };
 
 // One chunk slice of MMA tile TILE (16 rows): decode the lane's two blocks, four MMAs.
@@ -166,8 +166,9 @@ __global__ void __launch_bounds__(THREADS, 1) razer_direct_kernel(const Args a) 
   // this CTA's rows: a contiguous range of 16-row halves; a 32-row unit at either end may be shared with a neighbour
   int h_begin, h_end;
   if (a.unit_aligned) {
-    h_begin = 2 * blockIdx.x;
-    h_end = min(h_begin + 2, a.halves);
+    const int units = a.halves >> 1;
+    h_begin = 2 * (int)(((long long)units * blockIdx.x) / gridDim.x);
+    h_end = 2 * (int)(((long long)units * (blockIdx.x + 1)) / gridDim.x);
   } else {
     h_begin = (int)(((long long)a.halves * blockIdx.x) / gridDim.x);
     h_end = (int)(((long long)a.halves * (blockIdx.x + 1)) / gridDim.x);
@@ -371,22 +372,28 @@ struct DirectPlan {
   double balance;            // useful share of the SMs' time: rows are not split over K
 };
 
+// Rows go to CTAs either in whole 32-row units or in 16-row halves.  Halves balance better, but a unit shared
+// by two CTAs is walked by both, and every walk pays the per-chunk scaffolding again.  The busiest CTA's cost
+// per chunk, in instructions (measured: about 110 of scaffolding per walk, 104 per 16-row tile), decides.
 static DirectPlan direct_plan(const razer_desc* d) {
   const Geometry g = make_geometry(d->N, d->K);
   const int sms = direct_sm_count();
+  const double walk = 110.0, tile = 104.0;
   DirectPlan p;
-  p.halves = (g.row_tiles * TILE_ROWS) / 16;
-  const int units = (p.halves + 1) / 2;
-  if (units <= sms) {          // one whole 32-row unit per CTA: no unit is walked twice
-    p.grid = units;
-    p.unit_aligned = 1;
-    p.balance = (double)p.halves / (2.0 * sms);
-    return p;
+  p.halves = (g.row_tiles * TILE_ROWS) / 16;         // even: row tiles are 128 rows
+  const int units = p.halves / 2;
+  p.grid = units < sms ? units : sms;
+  const int units_max = (units + p.grid - 1) / p.grid;
+  const double cost_units = units_max * (walk + 2 * tile);
+  double cost_halves = cost_units;
+  if (units > sms) {
+    const int halves_max = (p.halves + sms - 1) / sms;
+    const int walks = halves_max / 2 + 1;            // worst case: a range that starts in the middle of a unit
+    cost_halves = walks * walk + halves_max * tile;
   }
-  p.grid = sms;
-  p.unit_aligned = 0;
-  const int per_cta = (p.halves + p.grid - 1) / p.grid;
-  p.balance = (double)p.halves / ((double)per_cta * sms);
+  p.unit_aligned = cost_units <= cost_halves ? 1 : 0;
+  const double cost = p.unit_aligned ? cost_units : cost_halves;
+  p.balance = p.halves * (tile + walk / 2) / (sms * cost);
   return p;
 }
 

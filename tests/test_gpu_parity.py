@@ -268,7 +268,7 @@ sys.path.insert(0, sys.argv[1])
 from oracle import razer_oracle as ro
 from paper_2501_04052_b200 import binding as b, inputs
 for (M, N, K, seed) in [(1, 1000, 4160, 1), (5, 333, 2064, 2), (16, 640, 1024, 3), (8, 384, 8192, 4), (2, 6000, 1088, 5),
-                        (1, 4096, 4096, 6)]:
+                        (1, 4096, 4096, 6), (3, 8200, 1024, 7)]:
     codes, scales = inputs.random_codes(N, K, seed=seed, scale_lo=0, scale_hi=64, zero_block_frac=0.02)
     codes, scales = codes.numpy(), scales.numpy()
     desc = b.make_desc(N, K, 0.004, sv_mag=(5.0, 9.0))
