@@ -11,8 +11,8 @@
 // weight-only kernel (weights pre-shuffled so that each thread's loads match its MMA fragment).
 //
 // Work unit: 32 weight rows (two 16-row MMA tiles) over the whole of K.  A CTA (16 warps) takes a contiguous
-// range of rows: whole units when there are no more units than SMs, else 16-row halves (a unit at either end
-// of the range may then be shared with the neighbouring CTA, each doing its own tile).  Inside a unit warp w
+// range of rows, in whole units or in 16-row halves, whichever the host's cost model prefers (with halves a unit
+// at either end of the range may be shared with the neighbouring CTA, each doing its own tile).  Inside a unit warp w
 // takes the chunks (64 columns) w, w + 16, ...  In a chunk, lane (g = lane / 4, t = lane % 4) decodes block t
 // of rows g and g + 8 of each tile; MMA q (0..3) takes elements 4q .. 4q + 3 of every lane's block, i.e. the
 // MMA's k slots are columns 16 t + 4 q + {0, 1, 2, 3}, for A and B alike.  At the end of a unit the 16 warps
