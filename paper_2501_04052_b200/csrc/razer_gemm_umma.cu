@@ -414,6 +414,8 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     constexpr int GROUPS = NDW / 4;
     static_assert(NDW % 4 == 0 && GROUPS <= ASTAGES, "every dequant group needs an A stage of its own");
     static_assert(!GI || (NACC % GROUPS == 0 && ASTAGES == GROUPS), "group issue: A stage and accumulators per group");
+    static_assert(GI ? STAGES % GROUPS == 0 : (GROUPS == ASTAGES && STAGES >= ASTAGES),
+                  "every fill of a stage must be known complete to the group that waits for the next one");
     constexpr int APG = GI ? NACC / GROUPS : NACC;       // accumulators per group
     // one warp of each group issues the group's MMAs; the groups pick different ones so that the issuing
     // warps sit on different schedulers (a warp's scheduler is warp % 4)
@@ -457,8 +459,18 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       if (turn == group) {
       const int astage = GI ? group : cur.astage;
       const uint32_t aph = GI ? own_phase : (uint32_t)cur.aphase;
-      if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 5)) break;
+      // Order matters.  A parity wait is only sound for a waiter that knows the barrier's previous phase to be
+      // complete, and a group does not see every fill of a shared-memory stage (the loads of a ring complete in
+      // any order: a group could come back to a stage one ring later while the fill it skipped is still in
+      // flight, take that for its own and decode the stage's old bytes).  Group issue: STAGES is a multiple of
+      // GROUPS, so a stage always serves the same group, which sees all its fills (making every group wait for
+      // the fills it skips is no way out: the groups free the stages themselves and end up waiting for one
+      // another).  Otherwise the A stage is
+      // this group's own (GROUPS == ASTAGES) and its release by the MMA warp, which takes the items in order,
+      // means that every item up to i - ASTAGES was issued, hence decoded, hence landed, the stage's previous
+      // fill (item i - STAGES, STAGES >= ASTAGES) among them.
       if (!wait_all(bar_aempty + 8 * astage, aph ^ 1u, 6)) break;
+      if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 5)) break;
       tc_fence_after();
       const uint32_t st = smem_addr(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
       const uint32_t a_t = tmem_a0 + astage * Cfg::A_STAGE_COLS + lane_off;
@@ -691,7 +703,7 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 3 : 1;
+  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -805,8 +817,8 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   switch (p.NT) {
     case 16:
       return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
-    case 32: return launch_cfg<32, 4, 5, 3, 12, 3, true>(tmap, a, p.grid, st);
-    case 64: return launch_cfg<64, 3, 5, 3, 12, 3, true>(tmap, a, p.grid, st);
+    case 32: return launch_cfg<32, 4, 6, 3, 12, 3, true>(tmap, a, p.grid, st);
+    case 64: return launch_cfg<64, 2, 8, 4, 16, 4, true>(tmap, a, p.grid, st);
     case 128: return launch_cfg<128, 1, 8, 4, 16, 1, false>(tmap, a, p.grid, st);
     default: return launch_cfg<256, 1, 5, 4, 16, 1, false>(tmap, a, p.grid, st);
   }

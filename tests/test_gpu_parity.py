@@ -224,6 +224,31 @@ def test_w4a4_config5_full_size_sampled_rows(b):
     assert err <= TOL, f"relative Frobenius error {err:.3e}"
 
 
+@pytest.mark.parametrize("M,N,K", [(2048, 14336, 4096), (64, 11008, 4096), (24, 4096, 11008)])
+def test_repeated_launches_are_bit_identical(b, M, N, K):
+    """The same call repeated many times must return the same bits.  The tcgen05 kernel once let a dequant
+    group mistake a weight load that was still in flight for the next load of the same stage (the loads of a
+    ring complete in any order, and a group does not watch the stages of the items it skips): about one launch
+    in a thousand of the first shape then produced a wrong partial tile at the start of a CTA's stripe."""
+    codes, scales = inputs.random_codes(N, K, seed=140)
+    desc, packed = _pack(b, codes.numpy(), scales.numpy(), 0.002)
+    x = inputs.activations(M, K, 141, outlier_channel_frac=0.01).cuda()
+    op, fn = (b.OP_GEMV, b.razer_gemv) if M <= 64 else (b.OP_GEMM, b.razer_gemm)
+    ws = b.alloc_workspace(desc, M, op, "cuda")
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    fn(desc, packed, x, y, ws)
+    first = y.clone()
+    differing = 0
+    for _ in range(1500):
+        fn(desc, packed, x, y, ws)
+        differing += int(not torch.equal(y, first))
+    b.razer_workspace_status(ws)
+    assert differing == 0, f"{differing} of 1500 launches differ from the first"
+    rows = sample_rows(N, 64, 142)
+    ref = ro.matmul_w4a16(inputs.bf16_to_bits(x.cpu()), codes.numpy()[rows], scales.numpy()[rows], np.float32(0.002))
+    assert rel_fro_bits(first[:, torch.from_numpy(rows).cuda()], ref) <= TOL
+
+
 # ------------------------------------------------------------------ host-buffer entry point, errors
 
 @pytest.mark.parametrize("pinned", [True, False])
