@@ -84,7 +84,12 @@ int razer_packed_bytes(const razer_desc* d, size_t* bytes_out);
  * N*K/16 bytes) and writes the packed form (razer_packed_bytes bytes, 16-byte aligned).
  * Inside the packed form the remapped code is always 0x8 and blocks whose special value is
  * positive are stored negated with a flag in the scale byte; both are lossless.
- * Asynchronous on `stream`. */
+ * Asynchronous on `stream`.
+ * The matmul entry points begin to read packed_dev before the single kernel directly ahead of
+ * them on the stream is known to have finished (programmatic dependent launch; RAZER_PDL=0 in
+ * the environment turns that off).  razer_pack_layout therefore queues an empty kernel behind
+ * its own, so its output is always safe to use; a caller that fills packed_dev with a kernel of
+ * its own must put some other operation between that kernel and the matmul. */
 int razer_pack_layout(const razer_desc* d, const uint8_t* codes_dev, const uint8_t* scales_dev,
                       void* packed_dev, void* stream);
 

@@ -129,13 +129,23 @@ static int grid_for(long long total, int threads) {
   return (int)(b < 1 ? 1 : (b > cap ? cap : b));
 }
 
+// The matmul kernels are launched with programmatic stream serialization and begin to fetch packed weights
+// before the kernel ahead of them in the stream is known to have finished (only activations, workspace and
+// outputs wait for it).  An empty, ordinarily launched kernel behind the pack kernel makes that kernel, not
+// the one that writes the weights, the matmul's predecessor: it cannot start before the weights are written
+// and visible.
+__global__ void pack_done_kernel() {}
+
 int launch_pack(const razer_desc* d, const uint8_t* codes, const uint8_t* scales, void* packed,
                 cudaStream_t st) {
   const Geometry g = make_geometry(d->N, d->K);
   const long long total = (long long)g.row_tiles * g.k_chunks * CHUNK_BLOCKS * TILE_ROWS;
   pack_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, scales, (uint8_t*)packed, g, d->remap_code);
   count_launches(1);
-  return check_cuda(cudaGetLastError(), "pack_kernel launch");
+  RAZER_TRY(check_cuda(cudaGetLastError(), "pack_kernel launch"));
+  pack_done_kernel<<<1, 32, 0, st>>>();
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "pack_done_kernel launch");
 }
 
 int launch_dequant(const razer_desc* d, const void* packed, void* out, int fp32, cudaStream_t st) {
