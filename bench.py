@@ -127,6 +127,21 @@ def make_sets(b, torch, inputs, N, K, n_sets, seed):
     return desc, sets, (codes, scales)
 
 
+def max_over_ranks(ms, dist, device):
+    """Slowest rank's time: the replicas are independent, so the job is as slow as its slowest GPU."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbps(world, step_bytes, ms):
+    """Aggregate over all replicas: every rank moves step_bytes per step in (at most) ms."""
+    return world * step_bytes / (ms * 1e-3) / 1e9
+
+
 def run_reference(args):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -230,11 +245,8 @@ def main():
     ms = time_cuda(lambda i: graph.replay(), 1, torch) / args.steps
     ms_stream = time_cuda(step, args.steps, torch)
     clocks = sampler.stop()
-    if dist:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * step_bytes / (ms * 1e-3) / 1e9
+    ms = max_over_ranks(ms, dist, "cuda")
+    value = whole_job_gbps(world, step_bytes, ms)
 
     # ---------------- end to end: host buffers, copies inside the timed region
     for l in layers:
@@ -249,11 +261,8 @@ def main():
         step_host(i)
     e2e_steps = max(20, args.steps // 4)
     ms_e2e = time_cuda(step_host, e2e_steps, torch)
-    if dist:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e = {"value": world * step_bytes / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s",
+    ms_e2e = max_over_ranks(ms_e2e, dist, "cuda")
+    e2e = {"value": whole_job_gbps(world, step_bytes, ms_e2e), "unit": "GB/s",
            "h2d_bytes_per_step": sum(2 * l["K"] for l in layers), "d2h_bytes_per_step": sum(2 * l["N"] for l in layers),
            "ms_per_step": ms_e2e}
 
