@@ -85,7 +85,7 @@ def _check_matmul(b, fn, desc, packed, codes, scales, d32, x, rows=None, **kw):
 
 
 def test_gemv_config1_student_t(b):
-    """BASELINE config 1: N=K=1024, Student-t x 0.02 weights from seed 0, M=1."""
+    """Workload config 1: N=K=1024, Student-t x 0.02 weights from seed 0, M=1."""
     w, codes, scales, d32 = oracle_quantized_weights(1024, 1024, 0, outliers=0.0)
     desc, packed = _pack(b, codes, scales, d32)
     x = inputs.activations(1, 1024, 0)
@@ -123,7 +123,7 @@ def test_gemv_other_special_values(b, sv_mag, remap_code):
 @pytest.mark.parametrize("M,N,K", [(4, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192),
                                    (4, 28672, 8192), (64, 28672, 8192), (16, 8192, 28672), (64, 8192, 28672)])
 def test_skinny_config3_full_size_sampled_rows(b, M, N, K):
-    """BASELINE config 3 at full size: random RaZeR codes, a sample of output columns checked
+    """Workload config 3 (skinny GEMM) at full size: random RaZeR codes, a sample of output columns checked
     one by one against the oracle."""
     codes, scales = inputs.random_codes(N, K, seed=40)
     codes, scales = codes.numpy(), scales.numpy()
@@ -196,7 +196,7 @@ def test_quant_act_given_scale_and_zero_input(b):
 
 @pytest.mark.parametrize("M,N,K", [(256, 1024, 8192), (17, 200, 464), (8, 300, 2048), (13, 520, 1040)])
 def test_w4a4_oracle_quantized(b, M, N, K):
-    """BASELINE config 5 (rows of N sampled down to keep the oracle quantizer quick)."""
+    """Workload config 5, W4A4 (rows of N sampled down to keep the oracle quantizer quick)."""
     w, wc, ws, wd = oracle_quantized_weights(N, K, 4)
     desc, packed = _pack(b, wc, ws, wd)
     x = inputs.activations(M, K, 90, outlier_channel_frac=0.01)
