@@ -356,6 +356,13 @@ def main():
         tf = 2.0 * M * N * K / (t * 1e-3) / 1e12
         extras.append({"config": 5, "op": "razer_gemm_w4a4", "M": M, "N": N, "K": K, "us": t * 1e3, "TFLOPs": tf,
                        "frac_bf16": tf / pk["bf16"]})
+        # GPU weight quantizer (offline step; FP32 in, interchange format out), 4096 x 4096
+        wq = inputs.student_t_weights(4096, 4096, 5000, outlier_frac=0.001).cuda()
+        b.razer_quant_weight(wq)
+        tw = graph_time(lambda i: b.razer_quant_weight(wq), 8)
+        extras.append({"config": "offline", "op": "razer_quant_weight", "N": 4096, "K": 4096, "us": tw * 1e3,
+                       "GBps": 4096 * 4096 * (4 + 0.5625) / (tw * 1e-3) / 1e9,
+                       "note": "bytes = one FP32 read + the 4.5-bit output; the kernel reads the input twice (maximum, then quantize)"})
         result["extras"] = extras
 
     if rank == 0 and not args.no_cpu:

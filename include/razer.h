@@ -170,6 +170,20 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag,
                     uint8_t* act_codes_dev, uint8_t* act_scales_dev,
                     float* tensor_scale_out_dev, void* stream);
 
+/* Weight quantizer on the GPU (Sec. 4.2, Eq. 1-3 and 6-7 with the 6-bit E3M3 block scale of
+ * Sec. 4.1): every block of 16 along K is quantized once per allowed special value, in
+ * metadata order +sv_mag[0], +sv_mag[1], -sv_mag[0], -sv_mag[1], and the lowest squared
+ * error wins (ties: the smaller metadata value).  w_dev: FP32 [N][K], K multiple of 16,
+ * 16-byte aligned.  tensor_scale_in_dev / amax_scratch_dev as in razer_quant_act.  Writes
+ * the interchange format that razer_pack_layout reads: codes_dev [N][K/2], scales_dev
+ * [N][K/16] ([meta(2) | E3M3 code(6)]), special value = remap_code (0x8 or 0x0), and the
+ * tensor scale to tensor_scale_out_dev.  Every FP32 step is a single IEEE operation in a
+ * fixed order, so the result is reproducible bit for bit.  Asynchronous on `stream`. */
+int razer_quant_weight(const float* w_dev, int N, int K, const float sv_mag[2], int remap_code,
+                       const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev,
+                       uint8_t* codes_dev, uint8_t* scales_dev, float* tensor_scale_out_dev,
+                       void* stream);
+
 /* Exact decode of RaZeR activations (interchange format, E4M3 scale, one metadata bit) to
  * bf16 [M][K] holding block_scale * element (the tensor scale is NOT applied). */
 int razer_decode_act(const uint8_t* act_codes_dev, const uint8_t* act_scales_dev, int M, int K,

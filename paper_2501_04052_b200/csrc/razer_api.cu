@@ -64,6 +64,8 @@ static int check_ptr(const void* p, size_t align, const char* name) {
 int launch_pack(const razer_desc*, const uint8_t*, const uint8_t*, void*, cudaStream_t);
 int launch_dequant(const razer_desc*, const void*, void*, int, cudaStream_t);
 int launch_decode_act(const uint8_t*, const uint8_t*, int, int, float, void*, cudaStream_t);
+int launch_quant_weight(const float*, int, int, float, float, int, const float*, uint32_t*, uint8_t*, uint8_t*,
+                        float*, cudaStream_t);
 int launch_quant_act(const void*, int, int, float, const float*, uint32_t*, uint8_t*, uint8_t*, float*,
                      cudaStream_t);
 int launch_gemv_simt(const razer_desc*, const void*, const void*, int, const float*, void*, void*, size_t,
@@ -274,6 +276,25 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag, const float* 
   if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 4, "amax_scratch_dev"));
   return launch_quant_act(x_dev, M, K, sv_mag, tensor_scale_in_dev, amax_scratch_dev, act_codes_dev,
                           act_scales_dev, tensor_scale_out_dev, (cudaStream_t)stream);
+}
+
+int razer_quant_weight(const float* w_dev, int N, int K, const float sv_mag[2], int remap_code,
+                       const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev, uint8_t* codes_dev,
+                       uint8_t* scales_dev, float* tensor_scale_out_dev, void* stream) {
+  if (N < 1 || K < 16 || K % 16) return set_error(RAZER_ERR_INVALID_ARG, "N=%d K=%d invalid (K %% 16 == 0)", N, K);
+  if (!sv_mag) return set_error(RAZER_ERR_INVALID_ARG, "sv_mag is NULL");
+  if (remap_code != 0x8 && remap_code != 0x0)
+    return set_error(RAZER_ERR_INVALID_ARG, "remap_code 0x%x is not a zero code", remap_code);
+  for (int i = 0; i < 2; ++i)
+    if (!sv_allowed(sv_mag[i]))
+      return set_error(RAZER_ERR_UNSUPPORTED, "special value magnitude %g is not allowed", sv_mag[i]);
+  RAZER_TRY(check_ptr(w_dev, 16, "w_dev"));
+  RAZER_TRY(check_ptr(codes_dev, 8, "codes_dev"));
+  RAZER_TRY(check_ptr(scales_dev, 1, "scales_dev"));
+  RAZER_TRY(check_ptr(tensor_scale_out_dev, 4, "tensor_scale_out_dev"));
+  if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 4, "amax_scratch_dev"));
+  return launch_quant_weight(w_dev, N, K, sv_mag[0], sv_mag[1], remap_code, tensor_scale_in_dev, amax_scratch_dev,
+                             codes_dev, scales_dev, tensor_scale_out_dev, (cudaStream_t)stream);
 }
 
 int razer_decode_act(const uint8_t* act_codes_dev, const uint8_t* act_scales_dev, int M, int K, float sv_mag,

@@ -128,6 +128,128 @@ __global__ void quant_act_kernel(const uint4* __restrict__ x, long long n_blocks
   }
 }
 
+// ------------------------------------------------------------------ offline weight quantizer (Sec. 4.2)
+// The same procedure as the activation quantizer above with the weight format: FP32 input, the 6-bit E3M3
+// block scale (codes 0..63 of the E4M3 grid, maximum 1.875) and four candidate special values
+// +m0, +m1, -m0, -m1 in metadata order (meta = sign * 2 + select, bits 7:6 of the scale byte).
+
+// Tensor maximum of |w| over FP32 input (Eq. 1 numerator); NaNs are skipped.
+__global__ void weight_amax_kernel(const float4* __restrict__ w, long long n_vec, uint32_t* __restrict__ amax_bits) {
+  uint32_t m = 0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 v = w[i];
+    const uint32_t b[4] = {__float_as_uint(v.x) & 0x7FFFFFFFu, __float_as_uint(v.y) & 0x7FFFFFFFu,
+                           __float_as_uint(v.z) & 0x7FFFFFFFu, __float_as_uint(v.w) & 0x7FFFFFFFu};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) m = max(m, (b[j] > 0x7F800000u) ? 0u : b[j]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  __shared__ uint32_t warp_max[32];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < (blockDim.x + 31) / 32 ? warp_max[threadIdx.x] : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (threadIdx.x == 0 && m) atomicMax(amax_bits, m);
+  }
+}
+
+// One thread per 16-element block.
+__global__ void quant_weight_kernel(const float4* __restrict__ w, long long n_blocks, float m0, float m1,
+                                    uint32_t remap_code, const float* __restrict__ scale_in,
+                                    const uint32_t* __restrict__ amax_bits, uint2* __restrict__ codes,
+                                    uint8_t* __restrict__ scales, float* __restrict__ scale_out) {
+  float d32;
+  if (scale_in) {
+    d32 = *scale_in;
+  } else {
+    const float amax = __uint_as_float(*amax_bits);
+    d32 = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, __fmul_rn(1.875f, 6.0f));   // Eq. 1
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = d32;
+  const float d32x6 = __fmul_rn(d32, 6.0f);
+  const uint32_t other_zero = remap_code ^ 8u;
+  const float cand[4] = {m0, m1, -m0, -m1};
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_blocks;
+       t += (long long)gridDim.x * blockDim.x) {
+    float xv[16];
+    float bmax = 0.0f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = w[4 * t + q];
+      xv[4 * q] = v.x, xv[4 * q + 1] = v.y, xv[4 * q + 2] = v.z, xv[4 * q + 3] = v.w;
+      bmax = fmaxf(bmax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+    uint32_t w0 = other_zero * 0x11111111u, w1 = w0, sbyte = 0;
+    if (bmax > 0.0f) {
+      const float tq = __fdiv_rn(bmax, d32x6);                         // Eq. 2 argument
+      uint32_t scode = round_to_e4m3(tq, 63u);
+      if (scode == 0) scode = 1;                                       // keep a non-empty block alive
+      const float denom = __fmul_rn(d32, scale_value(scode));
+      float err[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      uint32_t take[4] = {0, 0, 0, 0};
+      uint32_t std_lo = 0, std_hi = 0;                                 // plain FP4 codes, eight nibbles each
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float xs = __fdiv_rn(xv[j], denom);                      // the scaled block of Eq. 6
+        const uint32_t idx = round_to_fp4_idx(fabsf(xs));
+        const uint32_t neg = __float_as_uint(xs) >> 31;
+        const float r = neg ? -fp4_mag(idx) : fp4_mag(idx);
+        const float d_r = fabsf(__fsub_rn(xs, r));
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const bool tk = fabsf(__fsub_rn(xs, cand[c])) < d_r;         // strictly closer only
+          const float d = __fsub_rn(tk ? cand[c] : r, xs);
+          err[c] = __fadd_rn(err[c], __fmul_rn(d, d));                 // ascending j, no fusion
+          take[c] |= (uint32_t)tk << j;
+        }
+        const uint32_t sc = idx ? (idx | (neg << 3)) : other_zero;     // a true zero is always the other zero code
+        if (j < 8) std_lo |= sc << (4 * j); else std_hi |= sc << (4 * (j - 8));
+      }
+      uint32_t meta = 0;                                               // first minimum: ties keep the smaller metadata
+      float best = err[0];
+#pragma unroll
+      for (int c = 1; c < 4; ++c)
+        if (err[c] < best) { best = err[c]; meta = c; }
+      const uint32_t tk = take[0] * (meta == 0) | take[1] * (meta == 1) | take[2] * (meta == 2) | take[3] * (meta == 3);
+      w0 = std_lo, w1 = std_hi;
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if ((tk >> j) & 1u) {
+          if (j < 8) w0 = (w0 & ~(0xFu << (4 * j))) | (remap_code << (4 * j));
+          else w1 = (w1 & ~(0xFu << (4 * (j - 8)))) | (remap_code << (4 * (j - 8)));
+        }
+      sbyte = (meta << 6) | scode;
+    }
+    codes[t] = make_uint2(w0, w1);
+    scales[t] = (uint8_t)sbyte;
+  }
+}
+
+int launch_quant_weight(const float* w, int N, int K, float m0, float m1, int remap_code, const float* scale_in,
+                        uint32_t* amax_scratch, uint8_t* codes, uint8_t* scales, float* scale_out, cudaStream_t st) {
+  const long long n_blocks = (long long)N * (K / 16);
+  const long long n_vec = n_blocks * 4;
+  const int threads = 256;
+  if (!scale_in) {
+    RAZER_TRY(check_cuda(cudaMemsetAsync(amax_scratch, 0, sizeof(uint32_t), st), "amax memset"));
+    long long b = (n_vec + threads * 4 - 1) / (threads * 4);
+    const int g2 = (int)(b < 1 ? 1 : (b > 296 ? 296 : b));
+    weight_amax_kernel<<<g2, threads, 0, st>>>((const float4*)w, n_vec, amax_scratch);
+    count_launches(1);
+    RAZER_TRY(check_cuda(cudaGetLastError(), "weight_amax_kernel launch"));
+  }
+  long long b = (n_blocks + threads - 1) / threads;
+  const int g = (int)(b < 1 ? 1 : (b > 148LL * 16 ? 148LL * 16 : b));
+  quant_weight_kernel<<<g, threads, 0, st>>>((const float4*)w, n_blocks, m0, m1, (uint32_t)remap_code, scale_in,
+                                             amax_scratch, (uint2*)codes, scales, scale_out);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "quant_weight_kernel launch");
+}
+
 int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* scale_in,
                      uint32_t* amax_scratch, uint8_t* codes, uint8_t* scales, float* scale_out,
                      cudaStream_t st) {

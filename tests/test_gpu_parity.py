@@ -194,6 +194,47 @@ def test_quant_act_given_scale_and_zero_input(b):
     assert ts.item() == 1.0 and not codes.any() and not scales.any()
 
 
+@pytest.mark.parametrize("N,K,seed,sv_mag,remap_code", [(1024, 1024, 0, (5.0, 8.0), 0x8), (200, 80, 3, (5.0, 8.0), 0x8),
+                                                         (129, 4160, 5, (5.0, 9.0), 0x0), (300, 528, 6, (2.5, 12.0), 0x8)])
+def test_quant_weight_bit_exact(b, N, K, seed, sv_mag, remap_code):
+    """GPU weight quantizer against the oracle's (Sec. 4.2: E3M3 block scale, four special values): tensor scale,
+    scale codes, metadata and element codes, bit for bit except where two candidates' errors tie within rounding."""
+    w = inputs.student_t_weights(N, K, seed, outlier_frac=0.001)
+    codes, scales, ts = b.razer_quant_weight(w.cuda(), sv_mag=sv_mag, remap_code=remap_code)
+    torch.cuda.synchronize()
+    want_c, want_s, want_d, dbg = ro.quantize_weight(w.numpy(), sv_mag=sv_mag, remap_code=remap_code, return_debug=True)
+    assert np.float32(ts.item()) == want_d
+    got_s, got_c = scales.cpu().numpy(), codes.cpu().numpy()
+    assert np.array_equal(got_s & 0x3F, want_s & 0x3F)
+    blk_ok = (got_s == want_s) & np.all((got_c == want_c).reshape(N, K // 16, 8), axis=2)
+    assert np.all(blk_ok | dbg["near_tie"])
+    assert blk_ok.mean() > 0.999
+    # the GPU's codes go through the pack and dequant kernels like any others
+    desc, packed = _pack(b, got_c, got_s, float(ts.item()), sv_mag=sv_mag, remap_code=remap_code)
+    d2 = b.razer_dequant(desc, packed, fp32=True).cpu().numpy()
+    want2 = ro.dequant_d2(got_c, got_s, np.float32(ts.item()), sv_mag=sv_mag, remap_code=remap_code)
+    assert np.array_equal(d2.view(np.uint32), want2.view(np.uint32))
+    # and the quantization error is the format's: a few percent of the tensor's norm
+    assert np.linalg.norm(d2 - w.numpy()) / np.linalg.norm(w.numpy()) < 0.12
+
+
+def test_quant_weight_given_scale_and_zero_input(b):
+    w = inputs.student_t_weights(16, 256, 7)
+    given = torch.tensor([0.01], dtype=torch.float32)
+    codes, scales, ts = b.razer_quant_weight(w.cuda(), tensor_scale=given.cuda())
+    want_c, want_s, want_d = ro.quantize_weight(w.numpy(), tensor_scale=np.float32(0.01))
+    assert ts.item() == np.float32(0.01)
+    assert np.array_equal(scales.cpu().numpy(), want_s) and np.array_equal(codes.cpu().numpy(), want_c)
+    z = torch.zeros((4, 64), dtype=torch.float32)
+    codes, scales, ts = b.razer_quant_weight(z.cuda())
+    assert ts.item() == 1.0 and not codes.any() and not scales.any()
+    codes, scales, ts = b.razer_quant_weight(z.cuda(), remap_code=0x0)      # the true zero is then code 0x8
+    assert ts.item() == 1.0 and bool((codes == 0x88).all()) and not scales.any()
+    with pytest.raises(b.RazerError) as e:
+        b.razer_quant_weight(w.cuda(), sv_mag=(5.0, 6.0))                   # 6 is an FP4 value, not an allowed special value
+    assert e.value.code == b.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("M,N,K", [(256, 1024, 8192), (17, 200, 464), (8, 300, 2048), (13, 520, 1040)])
 def test_w4a4_oracle_quantized(b, M, N, K):
     """Workload config 5, W4A4 (rows of N sampled down to keep the oracle quantizer quick)."""
