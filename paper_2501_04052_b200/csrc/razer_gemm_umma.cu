@@ -234,8 +234,9 @@ struct ItemCursor {
 };
 
 // GI ("group issue"): each dequant group issues the MMAs of the items it decoded itself, into accumulators
-// of its own, instead of handing them to the MMA warp.  Used for narrow token tiles, where an item's MMAs
-// are short and one issuing warp per CTA would be the serial bottleneck.
+// of its own, instead of handing them to the MMA warp.  Used for the narrowest token tile (16), where an
+// item's MMAs are short; from 32 tokens up the MMA warp keeps up and issues (measured level at 16, the MMA
+// warp ahead at 32 and 64).
 template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC, bool GI>
 __global__ void __launch_bounds__(64 + 32 * NDW, 1)
 razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) {
@@ -425,8 +426,9 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     // Epilogue: with group issue only group 0 drains the (narrow) accumulators while the other groups
     // keep decoding; otherwise every group drains its share of the columns of its TMEM lane quarter.
     const bool epi_warp = !GI || (group == 0);
-    const int col_lo = GI ? 0 : group * (NT / GROUPS), col_hi = GI ? NT : col_lo + NT / GROUPS;
-    static_assert(GI || (NT / GROUPS) % 16 == 0, "epilogue column shares are multiples of 16");
+    // shares in units of 16 columns: group g takes units [g U / GROUPS, (g + 1) U / GROUPS), U = NT / 16
+    const int col_lo = GI ? 0 : 16 * ((group * (NT / 16)) / GROUPS);
+    const int col_hi = GI ? NT : 16 * (((group + 1) * (NT / 16)) / GROUPS);
     const bool leader = (threadIdx.x == 64);
     float ts = a.tensor_scale;                           // (x extra scale: read after the grid dependency)
     bool dep_waited = false;
@@ -703,7 +705,7 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  p.CH = p.NT <= 32 ? 4 : p.NT == 64 ? 2 : 1;
+  p.CH = p.NT <= 64 ? 4 : 1;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -817,8 +819,8 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   switch (p.NT) {
     case 16:
       return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
-    case 32: return launch_cfg<32, 4, 6, 3, 12, 3, true>(tmap, a, p.grid, st);
-    case 64: return launch_cfg<64, 2, 8, 4, 16, 4, true>(tmap, a, p.grid, st);
+    case 32: return launch_cfg<32, 4, 6, 3, 12, 2, false>(tmap, a, p.grid, st);
+    case 64: return launch_cfg<64, 4, 4, 3, 12, 2, false>(tmap, a, p.grid, st);
     case 128: return launch_cfg<128, 1, 8, 4, 16, 1, false>(tmap, a, p.grid, st);
     default: return launch_cfg<256, 1, 5, 4, 16, 1, false>(tmap, a, p.grid, st);
   }
