@@ -705,7 +705,7 @@ static UmmaPlan make_plan(const razer_desc* d, int M) {
   UmmaPlan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-  p.CH = p.NT <= 64 ? 4 : 1;
+  p.CH = p.NT <= 64 ? 4 : p.NT == 128 ? 2 : 1;
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.steps_per_tile = (g.k_chunks + p.CH - 1) / p.CH;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -821,7 +821,7 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
       return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
     case 32: return launch_cfg<32, 4, 6, 3, 12, 2, false>(tmap, a, p.grid, st);
     case 64: return launch_cfg<64, 4, 4, 3, 12, 2, false>(tmap, a, p.grid, st);
-    case 128: return launch_cfg<128, 1, 8, 4, 16, 1, false>(tmap, a, p.grid, st);
+    case 128: return launch_cfg<128, 2, 4, 4, 16, 1, false>(tmap, a, p.grid, st);
     default: return launch_cfg<256, 1, 5, 4, 16, 1, false>(tmap, a, p.grid, st);
   }
 }

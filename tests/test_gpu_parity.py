@@ -143,7 +143,8 @@ def test_skinny_config3_oracle_quantized(b):
 
 # ------------------------------------------------------------------ prefill GEMM
 
-@pytest.mark.parametrize("M,N,K", [(256, 512, 1024), (130, 200, 464), (2048, 1024, 4096)])
+@pytest.mark.parametrize("M,N,K", [(256, 512, 1024), (130, 200, 464), (2048, 1024, 4096), (100, 300, 1040),
+                                   (128, 640, 2048), (65, 129, 4160)])
 def test_gemm_oracle_quantized(b, M, N, K):
     w, codes, scales, d32 = oracle_quantized_weights(N, K, 3, outliers=0.0)
     desc, packed = _pack(b, codes, scales, d32)
@@ -265,7 +266,7 @@ def test_w4a4_config5_full_size_sampled_rows(b):
     assert err <= TOL, f"relative Frobenius error {err:.3e}"
 
 
-@pytest.mark.parametrize("M,N,K", [(2048, 14336, 4096), (64, 11008, 4096), (24, 4096, 11008)])
+@pytest.mark.parametrize("M,N,K", [(2048, 14336, 4096), (64, 11008, 4096), (24, 4096, 11008), (128, 11008, 4096)])
 def test_repeated_launches_are_bit_identical(b, M, N, K):
     """The same call repeated many times must return the same bits.  The tcgen05 kernel once let a dequant
     group mistake a weight load that was still in flight for the next load of the same stage (the loads of a
