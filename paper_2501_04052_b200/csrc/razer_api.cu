@@ -75,10 +75,6 @@ int launch_gemm_umma(const razer_desc*, const void* packed, const void* x, int M
                      const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
 size_t umma_workspace_bytes(const razer_desc*, int M);
 bool umma_supported(const razer_desc*, int M);
-int launch_gemv_mma(const razer_desc*, const void* packed, const void* x, int M, float extra_scale,
-                    const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
-size_t gemv_mma_workspace_bytes(const razer_desc*, int M);
-bool gemv_mma_supported(const razer_desc*, int M);
 int launch_gemv_direct(const razer_desc*, const void* packed, const void* x, int M, float extra_scale,
                        const float* extra_scale_dev, void* y, cudaStream_t);
 bool gemv_direct_supported(const razer_desc*, int M);
@@ -88,14 +84,12 @@ double gemv_direct_balance(const razer_desc*);
 // (razer_gemv_direct.cu) is faster whenever its fixed cost matters or the rows divide well over the SMs
 // (measured on B200: 5.1 against 12.7 us for 4096 x 4096, 47.7 against 50.0 at 8192 x 28672, level at 6144 x 28672,
 // 39.8 against 35.3 at 5120 x 28672 where its busiest CTA does 1.5 times the average), so it takes those shapes; with 9 to 16 tokens only the small ones.  RAZER_KERNEL (environment, read once) overrides: "umma" keeps
-// everything on the tcgen05 kernel, "direct" takes the register kernel wherever it is able to run, "mma"
-// routes M <= 16 to the older ring-fed mma.sync kernel (kept for comparison), "simt" routes everything to
-// the CUDA-core kernel (debugging aid).
+// everything on the tcgen05 kernel, "direct" takes the register kernel wherever it is able to run, "simt" routes
+// everything to the CUDA-core kernel (debugging aid).
 static char kernel_override() {
   static const char c = [] { const char* e = getenv("RAZER_KERNEL"); return e ? e[0] : '\0'; }();
   return c;
 }
-static bool use_mma(const razer_desc* d, int M) { return kernel_override() == 'm' && gemv_mma_supported(d, M); }
 static bool use_direct(const razer_desc* d, int M) {
   const char o = kernel_override();
   if (!gemv_direct_supported(d, M)) return false;
@@ -114,7 +108,6 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static size_t matmul_workspace_need(const razer_desc* d, int M) {
   size_t b = simt_workspace_bytes(d, M);
   if (umma_supported(d, M)) b = b > umma_workspace_bytes(d, M) ? b : umma_workspace_bytes(d, M);
-  if (gemv_mma_supported(d, M)) b = b > gemv_mma_workspace_bytes(d, M) ? b : gemv_mma_workspace_bytes(d, M);
   return b;
 }
 
@@ -208,8 +201,6 @@ static int matmul_common(const razer_desc* d, const void* packed_dev, const void
       return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
     return launch_gemv_direct(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, st);
   }
-  if (use_mma(d, M))
-    return launch_gemv_mma(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   if (umma_supported(d, M))
     return launch_gemm_umma(d, packed_dev, x_dev, M, d->K, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   razer_desc dd = *d;

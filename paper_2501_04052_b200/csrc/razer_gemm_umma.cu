@@ -195,6 +195,8 @@ struct UmmaArgs {
   long long total_items;
 };
 
+constexpr int MAX_ISSUERS = 5;          // the MMA warp, or one issuing warp per dequant group
+
 template <int NT, int CH, int STAGES, int ASTAGES, int NACC>
 struct UmmaCfg {
   static constexpr int W_BYTES = CH * CHUNK_BYTES;
@@ -207,7 +209,7 @@ struct UmmaCfg {
   static constexpr int TMEM_COLS_NEEDED = ACC_COLS + ASTAGES * A_STAGE_COLS;
   static constexpr int TMEM_COLS = TMEM_COLS_NEEDED <= 64 ? 64 : TMEM_COLS_NEEDED <= 128 ? 128
                                    : TMEM_COLS_NEEDED <= 256 ? 256 : 512;
-  static constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 3;
+  static constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 3 + MAX_ISSUERS;
   static constexpr int TABLE_BYTES = DECODE_TABLE_BYTES;        // scale table + special-value constants
   static constexpr size_t SMEM_BYTES =
       1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + NUM_BARS * 8 + 16 + 64 + TABLE_BYTES;
@@ -258,6 +260,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
   const uint32_t bar_accfull = bar_aempty + 8 * ASTAGES;
   const uint32_t bar_accempty = bar_accfull + 8;
   const uint32_t bar_epi = bar_accempty + 8;            // rendezvous of the 128 epilogue threads
+  const uint32_t bar_drain = bar_epi + 8;               // [MAX_ISSUERS] an issuing warp's own MMAs have all completed
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grid = gridDim.x, cta = blockIdx.x;
@@ -282,6 +285,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     mbar_init(bar_accfull, GI ? NDW / 4 : 1);
     mbar_init(bar_accempty, GI ? 128 : 32 * NDW);         // threads that read the accumulator in the epilogue
     mbar_init(bar_epi, GI ? 128 : 32 * NDW);
+    for (int i = 0; i < MAX_ISSUERS; ++i) mbar_init(bar_drain + 8 * i, 1);
     *abort_flag = 0;
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -349,6 +353,17 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     atomicCAS(a.status, 0u, code);
   };
 
+  // Whole warp, on leaving an issue loop (at its end or after a wait gave up): the MMAs this warp has issued
+  // read shared memory and TMEM and write TMEM until they complete, so the warp commits them to a barrier of
+  // its own and waits for it (bounded, not watching the abort flag) before the CTA may release either.
+  auto drain_mmas = [&](int issuer_idx) {
+    __syncwarp();
+    const uint32_t bar = bar_drain + 8 * issuer_idx;
+    if (elect_one()) tc_commit(bar);
+    __syncwarp();
+    mbar_wait(bar, 0u, tmem_slot + 3);
+  };
+
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
@@ -406,6 +421,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
         if (seg_last) ++seg;
         cur.template next<STAGES, ASTAGES>(spt);
       }
+      drain_mmas(0);
     }
   } else {
     // ===================== dequant (32 * NDW threads, thread = weight row) + epilogue =====================
@@ -414,6 +430,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     const int group = (warp - 2) >> 2;                   // four warps (all TMEM lane quarters) decode one item together
     constexpr int GROUPS = NDW / 4;
     static_assert(NDW % 4 == 0 && GROUPS <= ASTAGES, "every dequant group needs an A stage of its own");
+    static_assert(GROUPS + 1 <= MAX_ISSUERS, "a drain barrier per issuing warp");
     static_assert(!GI || (NACC % GROUPS == 0 && ASTAGES == GROUPS), "group issue: A stage and accumulators per group");
     static_assert(GI ? STAGES % GROUPS == 0 : (GROUPS == ASTAGES && STAGES >= ASTAGES),
                   "every fill of a stage must be known complete to the group that waits for the next one");
@@ -653,6 +670,7 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       }
       (void)it;
     }
+    if (GI && issuer) drain_mmas(1 + group);
   }
 
   tc_fence_before();

@@ -12,7 +12,8 @@ import torch
 from oracle import razer_oracle as ro
 from paper_2501_04052_b200 import inputs
 
-from _util import oracle_quantized_weights, rel_fro_bits, sample_rows, to_dev
+from _util import (elementwise_report, oracle_quantized_weights, oracle_reference, rel_fro_bits, rows_with_edge_tiles,
+                   sample_rows, to_dev)
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-3
@@ -65,6 +66,8 @@ def test_dequant_bit_exact_random_codes(b, remap_code, sv_mag):
 # ------------------------------------------------------------------ GEMV / skinny GEMM
 
 def _check_matmul(b, fn, desc, packed, codes, scales, d32, x, rows=None, **kw):
+    """Two calls on one workspace must agree bit for bit; the result must meet the relative Frobenius bar and,
+    element by element, lie within half a bf16 unit of the exact value plus the FP32 accumulation allowance."""
     op = b.OP_GEMV if fn is b.razer_gemv else b.OP_GEMM
     ws = b.alloc_workspace(desc, x.shape[0], op, "cuda")
     y = fn(desc, packed, x.cuda(), workspace=ws)
@@ -74,13 +77,17 @@ def _check_matmul(b, fn, desc, packed, codes, scales, d32, x, rows=None, **kw):
     assert torch.equal(y, y2), "second call with the same workspace differs"
     xb = inputs.bf16_to_bits(x)
     if rows is None:
-        ref = ro.matmul_w4a16(xb, codes, scales, np.float32(d32), **kw)
+        ref, y64, mag = oracle_reference(xb, codes, scales, np.float32(d32), **kw)
         got = y
     else:
-        ref = ro.matmul_w4a16(xb, codes[rows], scales[rows], np.float32(d32), **kw)
+        ref, y64, mag = oracle_reference(xb, codes[rows], scales[rows], np.float32(d32), **kw)
         got = y[:, torch.from_numpy(rows).cuda()]
     err = rel_fro_bits(got, ref)
     assert err <= TOL, f"relative Frobenius error {err:.3e}"
+    bad, differ, total = elementwise_report(got, ref, y64, mag)
+    print(f"[parity] {tuple(x.shape)} x {tuple(codes.shape)}: rel fro {err:.2e}, {differ} of {total} outputs differ from "
+          f"the oracle's bf16, {bad} outside the element-wise bound")
+    assert bad == 0, f"{bad} of {total} outputs outside 2^-8 |y| + 2^-20 sum|x w|"
     return err
 
 
@@ -121,7 +128,8 @@ def test_gemv_other_special_values(b, sv_mag, remap_code):
 
 
 @pytest.mark.parametrize("M,N,K", [(4, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192),
-                                   (4, 28672, 8192), (64, 28672, 8192), (16, 8192, 28672), (64, 8192, 28672)])
+                                   (4, 28672, 8192), (16, 28672, 8192), (4, 8192, 28672), (16, 8192, 28672),
+                                   (64, 8192, 28672)])
 def test_skinny_config3_full_size_sampled_rows(b, M, N, K):
     """Workload config 3 (skinny GEMM) at full size: random RaZeR codes, a sample of output columns checked
     one by one against the oracle."""
@@ -129,8 +137,19 @@ def test_skinny_config3_full_size_sampled_rows(b, M, N, K):
     codes, scales = codes.numpy(), scales.numpy()
     desc, packed = _pack(b, codes, scales, 0.002)
     x = inputs.activations(M, K, 40 + M)
-    rows = sample_rows(N, 192, 41)
+    rows = rows_with_edge_tiles(N, 192, 41)
     _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, 0.002, x, rows=rows)
+
+
+def test_skinny_config3_full_size_every_output(b):
+    """M = 64 against 28672 x 8192: every one of the 1.8 M outputs of the full-size launch is compared with the
+    oracle (computed in chunks of weight rows), so every CTA stripe and tile boundary is covered."""
+    M, N, K = 64, 28672, 8192
+    codes, scales = inputs.random_codes(N, K, seed=42)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.002)
+    x = inputs.activations(M, K, 43)
+    _check_matmul(b, b.razer_gemv, desc, packed, codes, scales, 0.002, x)
 
 
 def test_skinny_config3_oracle_quantized(b):
@@ -158,8 +177,18 @@ def test_gemm_config4_full_size_sampled_rows(b, N, K):
     codes, scales = codes.numpy(), scales.numpy()
     desc, packed = _pack(b, codes, scales, 0.002)
     x = inputs.activations(2048, K, 70, outlier_channel_frac=0.01)
-    rows = sample_rows(N, 96, 71)
+    rows = rows_with_edge_tiles(N, 96, 71)
     _check_matmul(b, b.razer_gemm, desc, packed, codes, scales, 0.002, x, rows=rows)
+
+
+def test_gemm_config4_full_size_every_output(b):
+    """M = 2048 against 4096 x 14336 (the shape whose stripes cut every output tile): all 8.4 M outputs."""
+    M, N, K = 2048, 4096, 14336
+    codes, scales = inputs.random_codes(N, K, seed=72)
+    codes, scales = codes.numpy(), scales.numpy()
+    desc, packed = _pack(b, codes, scales, 0.002)
+    x = inputs.activations(M, K, 73, outlier_channel_frac=0.01)
+    _check_matmul(b, b.razer_gemm, desc, packed, codes, scales, 0.002, x)
 
 
 # ------------------------------------------------------------------ activation quantization / W4A4
@@ -351,10 +380,10 @@ print("ok")
 """
 
 
-@pytest.mark.parametrize("kernel", ["umma", "direct", "mma", "simt"])
+@pytest.mark.parametrize("kernel", ["umma", "direct", "simt"])
 def test_alternative_kernels_match_the_oracle(kernel):
     """RAZER_KERNEL pins the matmul entry points to one kernel (the tcgen05 kernel, the register-only GEMV
-    kernel wherever it can run, the ring-fed mma.sync kernel, or the CUDA-core kernel) instead of the
+    kernel wherever it can run, or the CUDA-core kernel) instead of the
     per-shape choice; it is read once per process, so the check runs in a child process."""
     import os
     import subprocess
