@@ -197,6 +197,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-extras", action="store_true", help="skip the skinny / prefill / W4A4 lines")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--windows", type=int, default=7, help="timed windows (the median is reported)")
+    ap.add_argument("--window-ms", type=float, default=200.0, help="length of a timed window (0: one graph replay)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -258,10 +260,10 @@ def main():
     # about 200 ms, and the reported time per step is the median over 7 such windows (spread reported too); the
     # clock sampler runs across all of them.
     probe = time_cuda(lambda i: graph.replay(), 3, torch)                     # ms per replay
-    replays = max(1, int(200.0 / max(probe, 1e-3) + 0.5))
+    replays = max(1, int(args.window_ms / max(probe, 1e-3) + 0.5))
     sampler = ClockSampler(local_rank)
     sampler.start()
-    windows = [time_cuda(lambda i: graph.replay(), replays, torch) / args.steps for _ in range(7)]
+    windows = [time_cuda(lambda i: graph.replay(), replays, torch) / args.steps for _ in range(max(1, args.windows))]
     ms_stream = time_cuda(step, args.steps, torch)
     clocks = sampler.stop()
     windows.sort()

@@ -75,31 +75,30 @@ int launch_gemm_umma(const razer_desc*, const void* packed, const void* x, int M
                      const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
 size_t umma_workspace_bytes(const razer_desc*, int M);
 bool umma_supported(const razer_desc*, int M);
-int launch_gemv_direct(const razer_desc*, const void* packed, const void* x, int M, float extra_scale,
-                       const float* extra_scale_dev, void* y, cudaStream_t);
-bool gemv_direct_supported(const razer_desc*, int M);
-double gemv_direct_balance(const razer_desc*);
+int launch_gemv_stream(const razer_desc*, const void* packed, const void* x, int M, float extra_scale,
+                       const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
+size_t gemv_stream_workspace_bytes(const razer_desc*, int M);
+bool gemv_stream_supported(const razer_desc*, int M);
 
-// Kernel choice.  The tcgen05 kernel serves every M.  For M <= 16 the register-fragment kernel without split-K
-// (razer_gemv_direct.cu) is faster whenever its fixed cost matters or the rows divide well over the SMs
-// (measured on B200: 5.1 against 12.7 us for 4096 x 4096, 47.7 against 50.0 at 8192 x 28672, level at 6144 x 28672,
-// 39.8 against 35.3 at 5120 x 28672 where its busiest CTA does 1.5 times the average), so it takes those shapes; with 9 to 16 tokens only the small ones.  RAZER_KERNEL (environment, read once) overrides: "umma" keeps
-// everything on the tcgen05 kernel, "direct" takes the register kernel wherever it is able to run, "simt" routes
-// everything to the CUDA-core kernel (debugging aid).
+// Kernel choice.  M <= 8 (one group of tokens along the MMA's n) goes to the TMA-fed register-fragment kernel
+// (razer_gemv_stream.cu), whose fixed cost per launch is small and whose consumer warps do nothing but decode;
+// everything else to the tcgen05 kernel.  RAZER_KERNEL (environment, read once) overrides: "umma" keeps
+// everything on the tcgen05 kernel, "stream" is the default choice spelled out, "simt" routes everything to
+// the CUDA-core kernel (debugging aid).
 static char kernel_override() {
-  static const char c = [] { const char* e = getenv("RAZER_KERNEL"); return e ? e[0] : '\0'; }();
+  static const char c = [] {
+    const char* e = getenv("RAZER_KERNEL");
+    if (!e || !e[0]) return '\0';
+    if (e[0] == 's' && e[1] == 'i') return 's';         // simt
+    if (e[0] == 's') return 't';                        // stream
+    return e[0];                                        // umma
+  }();
   return c;
 }
-static bool use_direct(const razer_desc* d, int M) {
+static bool use_stream(const razer_desc* d, int M) {
   const char o = kernel_override();
-  if (!gemv_direct_supported(d, M)) return false;
-  if (o == 'd') return true;
-  if (o != '\0') return false;
-  const size_t bytes = make_geometry(d->N, d->K).packed_bytes();
-  // 9..16 tokens: a 32-row unit re-reads 1.8 times its own weight bytes of activations from L2, so only while
-  // the launch's fixed cost dominates (measured: 7.1 against 13.0 us at 4096 x 4096, 26.0 against 20.7 at 8192 x 8192)
-  if (M > 8) return bytes <= ((size_t)28 << 20);
-  return bytes <= ((size_t)64 << 20) || gemv_direct_balance(d) >= 0.8;
+  if (!gemv_stream_supported(d, M)) return false;
+  return o == '\0' || o == 't';
 }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -108,6 +107,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static size_t matmul_workspace_need(const razer_desc* d, int M) {
   size_t b = simt_workspace_bytes(d, M);
   if (umma_supported(d, M)) b = b > umma_workspace_bytes(d, M) ? b : umma_workspace_bytes(d, M);
+  if (gemv_stream_supported(d, M)) b = b > gemv_stream_workspace_bytes(d, M) ? b : gemv_stream_workspace_bytes(d, M);
   return b;
 }
 
@@ -194,13 +194,8 @@ static int matmul_common(const razer_desc* d, const void* packed_dev, const void
   RAZER_TRY(check_ptr(y_dev, 2, "y_dev"));
   if (ws && reinterpret_cast<uintptr_t>(ws) % 256)
     return set_error(RAZER_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
-  if (use_direct(d, M)) {
-    // this kernel needs no scratch, but the contract (a workspace of razer_workspace_bytes) is the same for every shape
-    const size_t need = matmul_workspace_need(d, M);
-    if (!ws || ws_bytes < need)
-      return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
-    return launch_gemv_direct(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, st);
-  }
+  if (use_stream(d, M))
+    return launch_gemv_stream(d, packed_dev, x_dev, M, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   if (umma_supported(d, M))
     return launch_gemm_umma(d, packed_dev, x_dev, M, d->K, extra_scale, extra_scale_dev, y_dev, ws, ws_bytes, st);
   razer_desc dd = *d;
@@ -250,8 +245,7 @@ int razer_gemv_host(const razer_desc* d, const void* packed_dev, const void* x_h
   if (y_target == y_stage_dev)
     RAZER_TRY(check_cuda(cudaMemcpyAsync(y_host, y_stage_dev, (size_t)M * d->N * 2, cudaMemcpyDeviceToHost, st),
                          "copy of y to the host"));
-  // the register-fragment kernel has no device-side wait that could give up: nothing to read back for it
-  if (workspace_dev && !use_direct(d, M)) return razer_workspace_status(workspace_dev, stream);   // synchronizes
+  if (workspace_dev) return razer_workspace_status(workspace_dev, stream);   // synchronizes
   return check_cuda(cudaStreamSynchronize(st), "stream synchronize");
 }
 

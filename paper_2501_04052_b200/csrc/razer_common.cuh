@@ -14,20 +14,23 @@ namespace razer {
 // ---------------------------------------------------------------------------------
 // Packed layout (GPU-internal form written by razer_pack_layout)
 //
-// The tensor is cut into tiles of TILE_ROWS rows x CHUNK_K columns (4 blocks of 16).
-// One tile-chunk is CHUNK_BYTES contiguous bytes:
-//   [blk 0..3][slot 0..127] 8 bytes: the block's 16 nibbles as two 32-bit words; row r sits in
-//                                    slot r for even blocks and r ^ 8 for odd ones (so that a
-//                                    warp reading rows g, g+1.. of four different blocks, the
-//                                    tensor-core fragment pattern, meets no bank conflict, while
-//                                    thread = row reads stay contiguous); element j of
-//                                    the block sits in word j/8, nibble (j%8)/2 + 4*(j%2), so
-//                                    that nibbles p and p+4 of a word (the same position in
-//                                    its two 16-bit halves) are elements 2p and 2p+1
-//   [row 0..127] 4 bytes           : the four blocks' scale bytes
-// so that thread = row reads are contiguous across a warp (8 B or 4 B stride) and a whole
-// chunk is one bulk copy.  Chunks are ordered [row tile][k chunk].  Rows beyond N and
-// columns beyond K are zero blocks (scale byte 0).
+// The tensor is cut into strips of STRIP_ROWS = 16 rows (one tensor-core row tile of the decode kernel) and
+// chunks of CHUNK_K = 64 columns (4 blocks of 16).  One strip-chunk ("piece") is PIECE_BYTES = 576 contiguous
+// bytes, and the pieces are ordered [strip][k chunk]: the whole K run of a strip is one contiguous byte range,
+// so any k range of any group of strips reaches shared memory with one bulk copy per strip.
+//   piece = [blk 0..3][slot 0..15] 8 bytes : the block's 16 nibbles as two 32-bit words; row r of the strip sits
+//                                            in slot r ^ (4 * blk), so that thread = row reads (16 consecutive
+//                                            slots) stay contiguous while the fragment-style read of the
+//                                            decode kernel (lane (g, t) reads rows g and g + 8 of block t)
+//                                            covers all banks; element j of the block sits in word j / 8,
+//                                            nibble (j % 8) / 2 + 4 * (j % 2), so that nibbles p and p + 4 of
+//                                            a word (the same position in its two 16-bit halves) are
+//                                            elements 2p and 2p + 1
+//           [g 0..7][blk 0..3][h 0..1] 1 byte : scale byte of row g + 8 h, block blk (the two bytes a lane
+//                                            of the decode kernel needs are adjacent; a row's four bytes
+//                                            sit in one 8-byte group)
+// Rows are padded to whole 128-row tiles (8 strips, what the tcgen05 kernel takes as one MMA tile) and columns
+// to whole chunks; rows beyond N and columns beyond K are zero blocks (scale byte 0).
 //
 // Inside the packed form:
 //   * the special value is always nibble 0x0, a true zero always nibble 0x8, every other
@@ -41,16 +44,21 @@ namespace razer {
 // is the one nibble that is numerically zero, and the block sign rides on the scale.
 // ---------------------------------------------------------------------------------
 constexpr int TILE_ROWS = 128;
+constexpr int STRIP_ROWS = 16;
+constexpr int TILE_STRIPS = TILE_ROWS / STRIP_ROWS;              // 8
 constexpr int CHUNK_K = 64;
 constexpr int CHUNK_BLOCKS = CHUNK_K / 16;
-constexpr int CHUNK_CODE_BYTES = CHUNK_BLOCKS * TILE_ROWS * 8;   // 4096
-constexpr int CHUNK_SCALE_BYTES = TILE_ROWS * 4;                 // 512
-constexpr int CHUNK_BYTES = CHUNK_CODE_BYTES + CHUNK_SCALE_BYTES;  // 4608
+constexpr int PIECE_CODE_BYTES = CHUNK_BLOCKS * STRIP_ROWS * 8;  // 512
+constexpr int PIECE_SCALE_BYTES = STRIP_ROWS * CHUNK_BLOCKS;     // 64
+constexpr int PIECE_BYTES = PIECE_CODE_BYTES + PIECE_SCALE_BYTES;   // 576
+constexpr int CHUNK_BYTES = TILE_STRIPS * PIECE_BYTES;           // 4608: one 128-row tile x 64 columns
 
 struct Geometry {
   int N, K;
   int row_tiles;   // ceil(N / 128)
   int k_chunks;    // ceil(K / 64)
+  __host__ __device__ int strips() const { return row_tiles * TILE_STRIPS; }
+  __host__ __device__ size_t strip_bytes() const { return (size_t)k_chunks * PIECE_BYTES; }   // one strip's K run
   __host__ __device__ size_t packed_bytes() const {
     return (size_t)row_tiles * (size_t)k_chunks * CHUNK_BYTES;
   }
@@ -64,6 +72,9 @@ __host__ __device__ inline Geometry make_geometry(int N, int K) {
   g.k_chunks = (K + CHUNK_K - 1) / CHUNK_K;
   return g;
 }
+
+// Every matmul workspace starts with the device status word (0 = ok), on a block of its own.
+constexpr size_t WS_STATUS_BYTES = 256;
 
 // Decode parameters derived from a razer_desc on the host, passed to kernels by value.
 struct DecodeParams {
@@ -108,10 +119,14 @@ __device__ __forceinline__ float scale_value(uint32_t code) {
   return e ? normal : (float)m * 0.001953125f;   // m * 2^-9
 }
 
-// Slot of row `row_in` (0..127) in block `blk` of a chunk, and the byte offset of its code words.
-__host__ __device__ __forceinline__ int packed_slot(int blk, int row_in) { return row_in ^ ((blk & 1) << 3); }
-__host__ __device__ __forceinline__ int packed_code_offset(int blk, int row_in) {
-  return (blk * TILE_ROWS + packed_slot(blk, row_in)) * 8;
+// Byte offsets inside a piece: the code words of row r (0..15) of block blk, and that block's scale byte.
+__host__ __device__ __forceinline__ int piece_code_offset(int blk, int r) { return (blk * STRIP_ROWS + (r ^ (4 * blk))) * 8; }
+__host__ __device__ __forceinline__ int piece_scale_offset(int blk, int r) {
+  return PIECE_CODE_BYTES + (r & 7) * 8 + blk * 2 + (r >> 3);
+}
+// Byte offset of the piece of (row n, k chunk c) in the packed buffer.
+__host__ __device__ __forceinline__ size_t piece_offset(const Geometry& g, int n, int c) {
+  return ((size_t)(n / STRIP_ROWS) * g.k_chunks + c) * PIECE_BYTES;
 }
 constexpr uint32_t PACKED_NEGATE = 0x40u, PACKED_SELECT = 0x80u;   // bits of a packed scale byte
 

@@ -5,8 +5,8 @@
 // Mapping onto the 5th-generation tensor core: the weight tile is the MMA's A operand
 // (128 weight rows = 128 TMEM lanes), the activation tile is the B operand (NT tokens,
 // K-major in shared memory, 128-byte swizzle, written by TMA), the accumulator D[128 x NT]
-// lives in TMEM.  Weights never exist as bf16 in shared or global memory: a TMA bulk copy
-// brings the packed 4.5-bit chunk into shared memory, the "dequant" warps (thread = weight
+// lives in TMEM.  Weights never exist as bf16 in shared or global memory: TMA bulk copies (one
+// per 16-row strip of the tile) bring the packed 4.5-bit chunks into shared memory, the "dequant" warps (thread = weight
 // row) decode one 16-element block at a time in registers and write the bf16 pairs straight
 // into TMEM with tcgen05.st, and the MMA reads A from TMEM.
 //
@@ -32,92 +32,15 @@
 
 #include "razer_common.cuh"
 #include "razer_decode.cuh"
+#include "razer_ptx.cuh"
 
 namespace razer {
 
 // ------------------------------------------------------------------ workspace layout
-constexpr size_t WS_STATUS_BYTES = 256;               // word 0: device status (0 = ok)
-constexpr uint32_t WAIT_LIMIT = 1u << 26;             // try_wait rounds before giving up, and
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;     // wall-clock bound of one wait (2 s)
 
 static size_t align256(size_t v) { return (v + 255) / 256 * 256; }
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// One poll of a barrier phase.  The hint lets the hardware park the thread until the phase
-// completes (or about the hinted time passes) instead of spinning in the issue slots that
-// the decoding warps need.
-constexpr uint32_t WAIT_SLICE_NS = 1000000u;
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(WAIT_SLICE_NS)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait; false = gave up (or another thread already flagged a failure).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();                     // only waits that already lasted a slice get here
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
-  }
-  return false;
-}
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-      "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
-      : "memory");
-}
-// True in exactly one lane of a converged warp.  Loops that only issue asynchronous work run
-// on the whole warp with this predicate around the issuing instructions, so that addresses
-// and descriptors stay warp-uniform values.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-  return pred != 0;
-}
-// Programmatic dependent launch: when the kernel was launched with the programmatic-serialization
-// attribute, `grid_dep_wait` returns once the preceding kernel in the stream has completed (otherwise at
-// once); everything that may depend on that kernel (activations, workspace, outputs) is touched after it,
-// while the weight stream, which depends on nothing, starts before.
-__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// ------------------------------------------------------------------ tcgen05 wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -241,7 +164,7 @@ struct ItemCursor {
 // warp ahead at 32 and 64).
 template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC, bool GI>
 __global__ void __launch_bounds__(64 + 32 * NDW, 1)
-razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) {
+razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const UmmaArgs a) {
   using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES, NACC>;
   constexpr int THREADS = 64 + 32 * NDW;
   extern __shared__ uint8_t smem_raw[];
@@ -312,14 +235,17 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
     const uint32_t bar = bar_full + 8 * cur.stage;
     const uint32_t n_x = a.x_map_3d ? CH : nch;           // the 3-D box always spans CH chunks (zero-filled past K)
-    mbar_expect_tx(bar, (uint32_t)(nch * CHUNK_BYTES) + n_x * Cfg::X_BOX_BYTES);
-    bulk_copy_g2s(st, a.packed + ((size_t)p_rt * a.g.k_chunks + c0) * CHUNK_BYTES, (uint32_t)(nch * CHUNK_BYTES), bar);
+    // The packed buffer as a (piece bytes, k chunk, strip) tensor: one box brings chunks c0 .. c0 + CH - 1 of the
+    // row tile's eight strips, [strip][chunk][piece] in shared memory (chunks past the end of K arrive as zeros).
+    mbar_expect_tx(bar, (uint32_t)(CH * CHUNK_BYTES) + n_x * Cfg::X_BOX_BYTES);
+    tma_load_3d(st, &tmap_w, 0, c0, p_rt * TILE_STRIPS, bar);
     if (with_x) produce_x(cur.stage, cur.step, p_tt);
     if (cur.step == spt - 1 && ++p_tt == a.token_tiles) { p_tt = 0; ++p_rt; }
     cur.template next<STAGES, ASTAGES>(spt);
   };
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_w) : "memory");
     grid_dep_launch();                                    // the next kernel may start its own prologue
     // first ring: packed weights now, their activation boxes once the preceding kernel has finished
     const ItemCursor first = cur;
@@ -464,6 +390,14 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
     };
     const DecodeTables dt = decode_tables_view(tables, lane);
     const uint32_t mul_lo = a.mul_lo, mul_hi = a.mul_hi;
+    // where this thread's weight row sits inside a stage: strip row / 16, row r = row % 16 of it
+    const int r16 = row % STRIP_ROWS;
+    const uint32_t strip_off = (uint32_t)(row / STRIP_ROWS) * (CH * PIECE_BYTES);
+    const uint32_t scale_off = (uint32_t)PIECE_CODE_BYTES + (uint32_t)(r16 & 7) * 8;
+    const uint32_t scale_sel = (r16 >> 3) ? 0x7531u : 0x6420u;
+    uint32_t code_off[CHUNK_BLOCKS];
+#pragma unroll
+    for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) code_off[blk] = (uint32_t)piece_code_offset(blk, r16);
     int turn = 0;                                        // item i is decoded by group i % GROUPS
     for (int i = 0; i < n_items; ++i, cur.template next<STAGES, ASTAGES>(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
       const int tile = cur.tile, step = cur.step;
@@ -491,17 +425,19 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const UmmaArgs a) 
       if (!wait_all(bar_aempty + 8 * astage, aph ^ 1u, 6)) break;
       if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 5)) break;
       tc_fence_after();
-      const uint32_t st = smem_addr(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES;
+      // this thread's strip of the stage: [strip 0..7][chunk 0..CH-1] pieces
+      const uint32_t st = smem_addr(smem) + (uint32_t)cur.stage * Cfg::STAGE_BYTES + strip_off;
       const uint32_t a_t = tmem_a0 + astage * Cfg::A_STAGE_COLS + lane_off;
 #pragma unroll
       for (int c = 0; c < CH; ++c) {
         if (c < nch) {
-          const uint32_t ck = st + c * CHUNK_BYTES;
+          const uint32_t ck = st + c * PIECE_BYTES;
           // all of the chunk's loads first, then the arithmetic
-          const uint32_t sw = lds32(ck + CHUNK_CODE_BYTES + row * 4);
+          const uint2 sq = lds64(ck + scale_off);           // the eight scale bytes of rows r % 8 and r % 8 + 8
+          const uint32_t sw = __byte_perm(sq.x, sq.y, scale_sel);   // this row's four, in block order
           uint2 cw[CHUNK_BLOCKS];
 #pragma unroll
-          for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) cw[blk] = lds64(ck + packed_code_offset(blk, row));
+          for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) cw[blk] = lds64(ck + code_off[blk]);
           uint32_t ss2[CHUNK_BLOCKS];
           SvConsts svc[CHUNK_BLOCKS];
 #pragma unroll
@@ -740,7 +676,7 @@ bool umma_supported(const razer_desc* d, int M) {
   (void)M;
   // RAZER_KERNEL=simt routes every matmul to the CUDA-core kernel (debugging aid)
   const char* e = getenv("RAZER_KERNEL");
-  return !(e && e[0] == 's');
+  return !(e && e[0] == 's' && e[1] == 'i');
 }
 
 size_t umma_workspace_bytes(const razer_desc* d, int M) {
@@ -756,7 +692,7 @@ size_t umma_workspace_zero_bytes(const razer_desc* d, int M) {
 }
 
 template <int NT, int CH, int STAGES, int ASTAGES, int NDW, int NACC, bool GI>
-static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, cudaStream_t st) {
+static int launch_cfg(const CUtensorMap& tmap, const CUtensorMap& tmap_w, const UmmaArgs& args, int grid, cudaStream_t st) {
   using Cfg = UmmaCfg<NT, CH, STAGES, ASTAGES, NACC>;
   auto kern = razer_umma_kernel<NT, CH, STAGES, ASTAGES, NDW, NACC, GI>;
   static bool attr_set = false;
@@ -778,7 +714,7 @@ static int launch_cfg(const CUtensorMap& tmap, const UmmaArgs& args, int grid, c
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap, args);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap, tmap_w, args);
   count_launches(1);
   return check_cuda(e, "razer_umma_kernel launch");
 }
@@ -815,6 +751,17 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
   if (r != CUDA_SUCCESS) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  // packed weights: (72 x 8 bytes of a piece, k chunk, strip), box = (whole piece, CH chunks, the tile's 8 strips)
+  CUtensorMap tmap_w;
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)(PIECE_BYTES / 8), (cuuint64_t)g.k_chunks, (cuuint64_t)g.strips()};
+    const cuuint64_t strides[2] = {(cuuint64_t)PIECE_BYTES, (cuuint64_t)g.strip_bytes()};
+    const cuuint32_t box[3] = {(cuuint32_t)(PIECE_BYTES / 8), (cuuint32_t)p.CH, (cuuint32_t)TILE_STRIPS};
+    r = enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_INT64, 3, const_cast<void*>(packed), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled (weights) failed with code %d", (int)r);
+  }
 
   UmmaArgs a;
   a.packed = (const uint8_t*)packed;
@@ -836,11 +783,11 @@ int launch_gemm_umma(const razer_desc* d, const void* packed, const void* x, int
   a.x_map_3d = map_3d;
   switch (p.NT) {
     case 16:
-      return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, a, p.grid, st);
-    case 32: return launch_cfg<32, 4, 6, 3, 12, 2, false>(tmap, a, p.grid, st);
-    case 64: return launch_cfg<64, 4, 4, 3, 12, 2, false>(tmap, a, p.grid, st);
-    case 128: return launch_cfg<128, 2, 4, 4, 16, 1, false>(tmap, a, p.grid, st);
-    default: return launch_cfg<256, 1, 5, 4, 16, 1, false>(tmap, a, p.grid, st);
+      return launch_cfg<16, 4, 6, 3, 12, 6, true>(tmap, tmap_w, a, p.grid, st);
+    case 32: return launch_cfg<32, 4, 6, 3, 12, 2, false>(tmap, tmap_w, a, p.grid, st);
+    case 64: return launch_cfg<64, 4, 4, 3, 12, 2, false>(tmap, tmap_w, a, p.grid, st);
+    case 128: return launch_cfg<128, 2, 4, 4, 16, 1, false>(tmap, tmap_w, a, p.grid, st);
+    default: return launch_cfg<256, 1, 5, 4, 16, 1, false>(tmap, tmap_w, a, p.grid, st);
   }
 }
 

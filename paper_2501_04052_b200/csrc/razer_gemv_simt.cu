@@ -38,12 +38,12 @@ gemv_simt_kernel(const uint8_t* __restrict__ packed, const __nv_bfloat16* __rest
     __syncthreads();
     const int c_lim = min(c_end, cg + SIMT_GROUP_CHUNKS);
     for (int c = cg; c < c_lim; ++c) {
-      const uint8_t* base = packed + ((size_t)rt * g.k_chunks + c) * CHUNK_BYTES;
-      const uint32_t sw = *reinterpret_cast<const uint32_t*>(base + CHUNK_CODE_BYTES + row_in * 4);
+      const uint8_t* base = packed + piece_offset(g, rt * TILE_ROWS + row_in, c);
+      const int r = row_in % STRIP_ROWS;
 #pragma unroll
       for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
-        const uint2 cw = *reinterpret_cast<const uint2*>(base + packed_code_offset(blk, row_in));
-        const uint32_t sb = (sw >> (8 * blk)) & 0xFFu;
+        const uint2 cw = *reinterpret_cast<const uint2*>(base + piece_code_offset(blk, r));
+        const uint32_t sb = base[piece_scale_offset(blk, r)];
         float s = scale_value(sb & 0x3Fu);
         if (sb & PACKED_NEGATE) s = -s;
         const float sv = (sb & PACKED_SELECT) ? sv1 : sv0;

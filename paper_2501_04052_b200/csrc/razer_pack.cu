@@ -49,9 +49,9 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __
     } else {
       w0 = w1 = 0x88888888u;                            // zero block: sixteen true zeros
     }
-    uint8_t* base = packed + (size_t)chunk * CHUNK_BYTES;
-    *reinterpret_cast<uint2*>(base + packed_code_offset(blk, row_in)) = make_uint2(w0, w1);
-    base[CHUNK_CODE_BYTES + row_in * 4 + blk] = (uint8_t)out_sb;
+    uint8_t* base = packed + piece_offset(g, n, kc);
+    *reinterpret_cast<uint2*>(base + piece_code_offset(blk, row_in % STRIP_ROWS)) = make_uint2(w0, w1);
+    base[piece_scale_offset(blk, row_in % STRIP_ROWS)] = (uint8_t)out_sb;
   }
 }
 
@@ -71,9 +71,9 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ packed, void* __restr
     const int n = rt * TILE_ROWS + row_in;
     const int k0 = (kc * CHUNK_BLOCKS + blk) * 16;
     if (n >= g.N || k0 >= g.K) continue;
-    const uint8_t* base = packed + (size_t)chunk * CHUNK_BYTES;
-    const uint2 c = *reinterpret_cast<const uint2*>(base + packed_code_offset(blk, row_in));
-    const uint32_t sb = base[CHUNK_CODE_BYTES + row_in * 4 + blk];
+    const uint8_t* base = packed + piece_offset(g, n, kc);
+    const uint2 c = *reinterpret_cast<const uint2*>(base + piece_code_offset(blk, row_in % STRIP_ROWS));
+    const uint32_t sb = base[piece_scale_offset(blk, row_in % STRIP_ROWS)];
     float s = scale_value(sb & 0x3Fu);
     if (sb & PACKED_NEGATE) s = -s;
     const float sv = p.sv_mag[(sb & PACKED_SELECT) ? 1 : 0];

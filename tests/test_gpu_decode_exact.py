@@ -71,7 +71,7 @@ def _run(kernel, Ms):
 
 @pytest.mark.parametrize("kernel,Ms", [
     ("", (1, 8, 16, 64)),                 # the kernels the library picks by itself for these sizes
-    ("direct", (1, 3, 8, 16)),            # register-fragment kernel: one and two token groups
+    ("stream", (1, 3, 8)),                # TMA-fed register-fragment kernel (M <= 8)
     ("umma", (16, 32, 64, 128, 256)),     # tcgen05 kernel: token tiles 16 (group issue), 32, 64, 128, 256
     ("simt", (1, 4)),                     # CUDA-core kernel
 ])

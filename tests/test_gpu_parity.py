@@ -380,10 +380,10 @@ print("ok")
 """
 
 
-@pytest.mark.parametrize("kernel", ["umma", "direct", "simt"])
+@pytest.mark.parametrize("kernel", ["umma", "stream", "simt"])
 def test_alternative_kernels_match_the_oracle(kernel):
-    """RAZER_KERNEL pins the matmul entry points to one kernel (the tcgen05 kernel, the register-only GEMV
-    kernel wherever it can run, or the CUDA-core kernel) instead of the
+    """RAZER_KERNEL pins the matmul entry points to one kernel (the tcgen05 kernel, the TMA-fed
+    register-fragment kernel wherever it can run (M <= 8), or the CUDA-core kernel) instead of the
     per-shape choice; it is read once per process, so the check runs in a child process."""
     import os
     import subprocess
