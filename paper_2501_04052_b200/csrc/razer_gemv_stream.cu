@@ -72,15 +72,15 @@ struct Args {
   const uint8_t* packed;
   const __nv_bfloat16* x;    // [M][K]
   __nv_bfloat16* y;          // [M][N]
-  float* slots;              // [grid][2][SLOT_FLOATS]
+  float* slots;              // [grid][SLOT_FLOATS]
   uint32_t* counters;        // one per split unit, zero between calls
   uint32_t* status;          // device status word
   const float* extra_scale;  // optional device scalar multiplied into the tensor scale
   int N, K, kc, M;
   int units;                 // units of TM strips that hold rows < N
   int whole_base, whole_per_cta;   // CTA b owns the whole units whole_base + b * whole_per_cta .. (clipped to units)
-  int rem_ctas;              // CTAs that share the split units [0, whole_base); 0 = nothing is split
-  uint32_t rem_slices;       // slices of the split units (rem_slices * grid < 2^32)
+  int rem_ctas;              // CTAs that share the split units [0, whole_base): pieces_per_unit each; 0 = nothing is split
+  int pieces_per_unit;       // a split unit is cut along K into this many equal pieces, one per CTA
   float sv0, sv1, tensor_scale;
   uint32_t mul_lo, mul_hi;   // 2^6 + 2^12 and 2^2 + 2^8 (razer_decode.cuh)
 };
@@ -124,18 +124,16 @@ struct Seg {
   int unit, c0, c1;
 };
 
-// A CTA's list of segments: at most two pieces of split units, then its whole units.
+// A CTA's list of segments: at most one piece of a split unit, then its whole units.
 struct Work {
   int n_rem, n_seg;
-  int u0, a0, a1;            // first split piece: unit, chunk range
-  int u1, b1;                // second split piece: unit, chunks [0, b1)
+  int u0, a0, a1;            // the piece of a split unit: unit, chunk range
   int wu0;                   // first whole unit
   int kc;
   __device__ __forceinline__ Seg seg(int i) const {
     Seg s;
     if (i < n_rem) {
-      if (i == 0) { s.unit = u0; s.c0 = a0; s.c1 = a1; }
-      else { s.unit = u1; s.c0 = 0; s.c1 = b1; }
+      s.unit = u0; s.c0 = a0; s.c1 = a1;
     } else {
       s.unit = wu0 + (i - n_rem);
       s.c0 = 0;
@@ -149,27 +147,20 @@ __device__ __forceinline__ Work make_work(const Args& a, int b) {
   Work w;
   w.kc = a.kc;
   w.n_rem = 0;
-  w.u0 = w.a0 = w.a1 = w.u1 = w.b1 = 0;
+  w.u0 = w.a0 = w.a1 = 0;
   if (b < a.rem_ctas) {
-    const uint32_t s0 = (a.rem_slices * (uint32_t)b) / (uint32_t)a.rem_ctas;
-    const uint32_t s1 = (a.rem_slices * (uint32_t)(b + 1)) / (uint32_t)a.rem_ctas;   // s1 > s0
-    w.u0 = (int)(s0 / (uint32_t)a.kc);
-    w.u1 = (int)((s1 - 1) / (uint32_t)a.kc);
-    w.a0 = (int)s0 - w.u0 * a.kc;
-    w.n_rem = w.u1 > w.u0 ? 2 : 1;
-    w.a1 = w.n_rem == 2 ? a.kc : (int)s1 - w.u0 * a.kc;
-    w.b1 = (int)s1 - w.u1 * a.kc;
+    // piece j of unit u: chunks [kc j / p, kc (j + 1) / p)
+    w.u0 = b / a.pieces_per_unit;
+    const int j = b - w.u0 * a.pieces_per_unit;
+    w.a0 = (a.kc * j) / a.pieces_per_unit;
+    w.a1 = (a.kc * (j + 1)) / a.pieces_per_unit;
+    w.n_rem = 1;
   }
   w.wu0 = a.whole_base + b * a.whole_per_cta;
   int n_whole = a.units - w.wu0;
   n_whole = n_whole < 0 ? 0 : (n_whole > a.whole_per_cta ? a.whole_per_cta : n_whole);
   w.n_seg = w.n_rem + n_whole;
   return w;
-}
-
-// CTA that owns slice s of the split units (the inverse of the range formula in make_work).
-__device__ __forceinline__ int cta_of_slice(uint32_t s, int ctas, uint32_t total) {
-  return (int)((((s + 1u) * (uint32_t)ctas) - 1u) / total);
 }
 
 // Four stored nibbles of each 16-bit half of `w` -> four bf16x2 registers (elements 2p, 2p + 1 of the word in
@@ -438,21 +429,19 @@ __global__ void __launch_bounds__(THREADS, OCC) razer_stream_kernel(const Args a
         continue;
       }
       // ---- a piece of a split unit: publish, count, the last arrival adds the pieces in CTA order ----
-      float* mine = a.slots + ((size_t)b * 2 + i) * SLOT_FLOATS;
+      float* mine = a.slots + (size_t)b * SLOT_FLOATS;
 #pragma unroll
       for (int j = 0; j < MAX_M; ++j)
         if (lane + 32 * j < outputs) mine[lane + 32 * j] = v[j];
       __syncwarp();
-      const uint32_t u_begin = (uint32_t)s.unit * (uint32_t)a.kc;
-      const int c_first = cta_of_slice(u_begin, a.rem_ctas, a.rem_slices);
-      const int c_last = cta_of_slice(u_begin + a.kc - 1, a.rem_ctas, a.rem_slices);
+      const int c_first = s.unit * a.pieces_per_unit, c_last = c_first + a.pieces_per_unit - 1;
       uint32_t last = 0;
       if (lane == 0) {
         uint32_t prev;
         // release: this warp's slot stores (ordered before by the warp barrier) become visible with the count;
         // acquire: the last arrival sees every earlier arrival's slot stores
         asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.counters + s.unit) : "memory");
-        last = (prev + 1 == (uint32_t)(c_last - c_first + 1)) ? 1u : 0u;
+        last = (prev + 1 == (uint32_t)a.pieces_per_unit) ? 1u : 0u;
         if (last) a.counters[s.unit] = 0;                     // leave the counter ready for the next call
       }
       last = __shfl_sync(0xFFFFFFFFu, last, 0);
@@ -462,20 +451,12 @@ __global__ void __launch_bounds__(THREADS, OCC) razer_stream_kernel(const Args a
       for (int j = 0; j < MAX_M; ++j) acc[j] = 0.0f;
       // CTA order (a fixed summation order); the loads of four CTAs' slots are in flight together
       for (int cb = c_first; cb <= c_last; cb += 4) {
-        const float* src[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int c = min(cb + u, c_last);
-          const uint32_t c_start = (a.rem_slices * (uint32_t)c) / (uint32_t)a.rem_ctas;
-          const int sl = (int)(c_start / (uint32_t)a.kc) == s.unit ? 0 : 1;     // the unit is that CTA's first or second piece
-          src[u] = a.slots + ((size_t)c * 2 + sl) * SLOT_FLOATS;
-        }
 #pragma unroll
         for (int j = 0; j < MAX_M; ++j) {
           if (lane + 32 * j < outputs) {
             float part[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) part[u] = __ldcg(src[u] + lane + 32 * j);
+            for (int u = 0; u < 4; ++u) part[u] = __ldcg(a.slots + (size_t)min(cb + u, c_last) * SLOT_FLOATS + lane + 32 * j);
 #pragma unroll
             for (int u = 0; u < 4; ++u)
               if (cb + u <= c_last) acc[j] += part[u];
@@ -592,59 +573,78 @@ static int stream_sm_count() {
 
 struct StreamPlan {
   int TM, SPW, grid, units, kc;
-  int whole_base, whole_per_cta, rem_ctas;
-  uint32_t rem_slices;
+  int whole_base, whole_per_cta, rem_ctas, pieces_per_unit;
+  double cost;
   size_t counters_bytes, slots_bytes;
 };
 
 static size_t align256s(size_t v) { return (v + 255) / 256 * 256; }
 
-// Whole units only, or q whole units per CTA plus the remaining units cut along K (processed first, combined
-// through the workspace).  Costs are slices on the busiest CTA; when nothing follows the split part (q == 0)
-// its combination is exposed at the end of the launch, which costs about as much as 40 strip-slices.
-static StreamPlan stream_plan(const razer_desc* d, int M) {
+// One candidate: units of TM strips; every CTA takes whole units only (split == false), or q whole units after a
+// piece of one of the remaining units, each of which is cut along K into equal pieces (processed first, combined
+// through the workspace).  The cost is the busiest CTA's work in strip-slices: a slice of TM strips costs TM plus
+// what is per slice (activation fragment, loop), and a split whose combination nothing follows (q == 0) pays
+// for it at the end of the launch.
+static StreamPlan stream_candidate(const razer_desc* d, int M, int G, int TM, bool split) {
   using namespace stream_path;
   StreamPlan p;
   const Geometry g = make_geometry(d->N, d->K);
-  static const int per_sm = [] { const char* e = getenv("RAZER_STREAM_CTAS"); const int v = e ? atoi(e) : 0; return v >= 1 && v <= OCC ? v : OCC; }();   // tuning aid
-  const int G = per_sm * stream_sm_count();
   const int strips = (d->N + STRIP_ROWS - 1) / STRIP_ROWS;
-  p.TM = ((strips + 1) / 2 >= G) ? 2 : 1;
-  p.units = (strips + p.TM - 1) / p.TM;
+  p.TM = TM;
+  p.units = (strips + TM - 1) / TM;
   p.kc = g.k_chunks;
   // slices per warp and stage: as many as leave three stages in what a CTA has for its ring
   p.SPW = 1;
   const int ring_bytes = SMEM_BYTES - TABLE_BYTES - 2 * CW * M * RED_STRIDE * 4 - 2048;
-  for (int spw = (p.TM == 1 ? 4 : 2); spw >= 1; spw >>= 1) {
-    const int stage = p.TM * CW * spw * PIECE_BYTES + M * (CW * spw * 128 + 16);
+  for (int spw = (TM == 1 ? 4 : 2); spw >= 1; spw >>= 1) {
+    const int stage = TM * CW * spw * PIECE_BYTES + M * (CW * spw * 128 + 16);
     if (3 * stage <= ring_bytes) { p.SPW = spw; break; }
   }
+  const double per_slice = TM + 0.12 + 0.04 * M;
   const int q = p.units / G, rem = p.units - q * G;
-  const long long R = (long long)rem * p.kc;
-  // at least one CTA per split unit, so that no range spans more than two units; at least a stage's worth of slices each
-  const int Gr = rem ? (int)std::max<long long>(rem, std::min<long long>(G, R / CW)) : 0;
-  const long long cost_split = (long long)q * p.kc + (Gr ? (R + Gr - 1) / Gr : 0) + (q == 0 ? 40 / p.TM : 0);
-  const int qa = (p.units + G - 1) / G;
-  const long long cost_whole = (long long)qa * p.kc;
-  static const char force = [] { const char* e = getenv("RAZER_STREAM_SPLIT"); return e ? e[0] : '\0'; }();   // '0' / '1': tuning aid
-  const bool fits32 = R * (long long)(G + 1) < (1ll << 32);            // the kernel's slice arithmetic is 32-bit
-  const bool split = fits32 && (force == '1' ? rem > 0 : force == '0' ? false : (rem > 0 && cost_split < cost_whole));
-  if (split) {
+  if (split && rem > 0) {
+    int pieces = G / rem;                                               // >= 1
+    pieces = std::max(1, std::min(pieces, p.kc / CW));                  // a piece is at least one slice per warp
     p.whole_base = rem;
     p.whole_per_cta = q;
-    p.rem_ctas = Gr;
-    p.rem_slices = (uint32_t)R;
-    p.grid = q > 0 ? G : Gr;
+    p.pieces_per_unit = pieces;
+    p.rem_ctas = rem * pieces;
+    p.grid = q > 0 ? G : p.rem_ctas;
+    p.cost = ((double)q * p.kc + (p.kc + pieces - 1) / pieces) * per_slice + (q == 0 && pieces > 1 ? 40.0 : 0.0);
   } else {
+    const int qa = (p.units + G - 1) / G;
     p.whole_base = 0;
     p.whole_per_cta = qa;
+    p.pieces_per_unit = 1;
     p.rem_ctas = 0;
-    p.rem_slices = 0;
     p.grid = (p.units + qa - 1) / qa;
+    p.cost = (double)qa * p.kc * per_slice;
   }
   p.counters_bytes = align256s((size_t)G * sizeof(uint32_t));           // at most G - 1 split units
-  p.slots_bytes = (size_t)G * 2 * SLOT_FLOATS * sizeof(float);
+  p.slots_bytes = (size_t)G * SLOT_FLOATS * sizeof(float);
   return p;
+}
+
+// The cheapest of the four candidates (one or two strips per unit, with or without a split).
+static StreamPlan stream_plan(const razer_desc* d, int M) {
+  using namespace stream_path;
+  static const int per_sm = [] { const char* e = getenv("RAZER_STREAM_CTAS"); const int v = e ? atoi(e) : 0; return v >= 1 && v <= OCC ? v : OCC; }();   // tuning aids
+  static const char force_split = [] { const char* e = getenv("RAZER_STREAM_SPLIT"); return e ? e[0] : '\0'; }();
+  static const char force_tm = [] { const char* e = getenv("RAZER_STREAM_TM"); return e ? e[0] : '\0'; }();
+  const int G = per_sm * stream_sm_count();
+  StreamPlan best;
+  bool have = false;
+  for (int TM = 1; TM <= 2; ++TM) {
+    if ((force_tm == '1' && TM != 1) || (force_tm == '2' && TM != 2)) continue;
+    for (int split = 0; split <= 1; ++split) {
+      if (force_split == '0' && split) continue;
+      const StreamPlan c = stream_candidate(d, M, G, TM, split != 0);
+      if (force_split == '1' && !split && c.units % G != 0) continue;
+      if (!have || c.cost < best.cost) { best = c; have = true; }
+    }
+  }
+  if (!have) best = stream_candidate(d, M, G, 1, false);
+  return best;
 }
 
 bool gemv_stream_supported(const razer_desc* d, int M) {
@@ -704,7 +704,7 @@ int launch_gemv_stream(const razer_desc* d, const void* packed, const void* x, i
   a.whole_base = p.whole_base;
   a.whole_per_cta = p.whole_per_cta;
   a.rem_ctas = p.rem_ctas;
-  a.rem_slices = p.rem_slices;
+  a.pieces_per_unit = p.pieces_per_unit;
   a.sv0 = d->sv_mag[0];
   a.sv1 = d->sv_mag[1];
   a.tensor_scale = d->tensor_scale * extra_scale;

@@ -364,7 +364,7 @@ sys.path.insert(0, sys.argv[1])
 from oracle import razer_oracle as ro
 from paper_2501_04052_b200 import binding as b, inputs
 for (M, N, K, seed) in [(1, 1000, 4160, 1), (5, 333, 2064, 2), (16, 640, 1024, 3), (8, 384, 8192, 4), (2, 6000, 1088, 5),
-                        (1, 4096, 4096, 6), (3, 8200, 1024, 7)]:
+                        (1, 4096, 4096, 6), (3, 8200, 1024, 7), (2, 11008, 2048, 8), (1, 50, 16, 9), (8, 5000, 144, 10)]:
     codes, scales = inputs.random_codes(N, K, seed=seed, scale_lo=0, scale_hi=64, zero_block_frac=0.02)
     codes, scales = codes.numpy(), scales.numpy()
     desc = b.make_desc(N, K, 0.004, sv_mag=(5.0, 9.0))
@@ -380,8 +380,16 @@ print("ok")
 """
 
 
-@pytest.mark.parametrize("kernel", ["umma", "stream", "simt"])
-def test_alternative_kernels_match_the_oracle(kernel):
+@pytest.mark.parametrize("kernel,extra_env", [
+    ("umma", {}), ("simt", {}), ("stream", {}),
+    # the decode kernel's partitions, each forced on every shape: whole units only / units cut along K and combined
+    # through the workspace, with one or two 16-row strips per unit
+    ("stream", {"RAZER_STREAM_SPLIT": "0", "RAZER_STREAM_TM": "1"}),
+    ("stream", {"RAZER_STREAM_SPLIT": "0", "RAZER_STREAM_TM": "2"}),
+    ("stream", {"RAZER_STREAM_SPLIT": "1", "RAZER_STREAM_TM": "1"}),
+    ("stream", {"RAZER_STREAM_SPLIT": "1", "RAZER_STREAM_TM": "2"}),
+])
+def test_alternative_kernels_match_the_oracle(kernel, extra_env):
     """RAZER_KERNEL pins the matmul entry points to one kernel (the tcgen05 kernel, the TMA-fed
     register-fragment kernel wherever it can run (M <= 8), or the CUDA-core kernel) instead of the
     per-shape choice; it is read once per process, so the check runs in a child process."""
@@ -389,7 +397,7 @@ def test_alternative_kernels_match_the_oracle(kernel):
     import subprocess
     import sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    env = dict(os.environ, RAZER_KERNEL=kernel)
+    env = dict(os.environ, RAZER_KERNEL=kernel, **extra_env)
     r = subprocess.run([sys.executable, "-c", _ALT_KERNEL_CHECK, root], env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "ok" in r.stdout, r.stdout + r.stderr
 
