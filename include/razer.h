@@ -162,9 +162,14 @@ int razer_gemv_static(const razer_desc* d, const void* packed_dev, const void* x
  * special value, +sv_mag and -sv_mag, and the lower squared error wins; Eq. 1-3, 6-7 with
  * the 7-bit E4M3 block scale).  x_dev: bf16 [M][K], K multiple of 16.
  * tensor_scale_in_dev: device float to use as the Eq. 1 scale, or NULL to compute it from
- * the tensor maximum (then amax_scratch_dev, one device uint32, is required and is
- * overwritten).  Writes act_codes_dev [M][K/2], act_scales_dev [M][K/16] in the
- * interchange format (remapped code 0x8) and the scale used to tensor_scale_out_dev. */
+ * the tensor maximum.  In that case amax_scratch_dev is required: two device uint32 (8-byte
+ * aligned) that are ZERO before the first call; every call leaves them zero again, so one
+ * scratch serves any number of calls one after another (calls that may overlap on the GPU
+ * need a scratch each; after a call that was interrupted mid-kernel clear it again).  The
+ * whole call is one kernel launch; with a computed scale its CTAs meet once (cooperative
+ * launch), and a scale of NaN in tensor_scale_out_dev reports a scratch that was not zero.
+ * Writes act_codes_dev [M][K/2], act_scales_dev [M][K/16] in the interchange format
+ * (remapped code 0x8) and the scale used to tensor_scale_out_dev. */
 int razer_quant_act(const void* x_dev, int M, int K, float sv_mag,
                     const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev,
                     uint8_t* act_codes_dev, uint8_t* act_scales_dev,

@@ -194,14 +194,22 @@ def razer_gemv_host(desc, packed, x_host, y_host, x_stage, y_stage, workspace) -
                                 _ptr(y_stage), _ptr(workspace), workspace.numel(), _stream()))
 
 
-def razer_quant_act(x: torch.Tensor, sv_mag: float = 5.0, tensor_scale: torch.Tensor | None = None):
-    """x bf16 [M, K] (device) -> (codes uint8 [M, K/2], scales uint8 [M, K/16], tensor scale float32 [1])."""
+_quant_act_scratch = {}
+
+
+def razer_quant_act(x: torch.Tensor, sv_mag: float = 5.0, tensor_scale: torch.Tensor | None = None,
+                    scratch: torch.Tensor | None = None):
+    """x bf16 [M, K] (device) -> (codes uint8 [M, K/2], scales uint8 [M, K/16], tensor scale float32 [1]).
+    `scratch`: two zeroed int32 on the device (left zero by every call); one per device is kept here when none is given."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
     M, K = x.shape
     codes = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
     scales = torch.empty((M, K // 16), dtype=torch.uint8, device=x.device)
     out_scale = torch.empty(1, dtype=torch.float32, device=x.device)
-    scratch = torch.empty(1, dtype=torch.int32, device=x.device)
+    if scratch is None:
+        scratch = _quant_act_scratch.get(x.device)
+        if scratch is None:
+            scratch = _quant_act_scratch[x.device] = torch.zeros(2, dtype=torch.int32, device=x.device)
     _check(_lib.razer_quant_act(_ptr(x), M, K, float(sv_mag), _ptr(tensor_scale), _ptr(scratch), _ptr(codes),
                                 _ptr(scales), _ptr(out_scale), _stream()))
     return codes, scales, out_scale

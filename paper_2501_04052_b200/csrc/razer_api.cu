@@ -258,7 +258,7 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag, const float* 
   RAZER_TRY(check_ptr(act_codes_dev, 8, "act_codes_dev"));
   RAZER_TRY(check_ptr(act_scales_dev, 1, "act_scales_dev"));
   RAZER_TRY(check_ptr(tensor_scale_out_dev, 4, "tensor_scale_out_dev"));
-  if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 4, "amax_scratch_dev"));
+  if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 8, "amax_scratch_dev"));
   return launch_quant_act(x_dev, M, K, sv_mag, tensor_scale_in_dev, amax_scratch_dev, act_codes_dev,
                           act_scales_dev, tensor_scale_out_dev, (cudaStream_t)stream);
 }

@@ -8,36 +8,6 @@
 
 namespace razer {
 
-// Tensor maximum of |x| (Eq. 1 numerator): bit patterns of non-negative floats order like
-// unsigned integers, so one atomicMax per warp on the bf16 magnitude pattern suffices.
-__global__ void act_amax_kernel(const uint4* __restrict__ x, long long n_vec, uint32_t* __restrict__ amax_bits) {
-  uint32_t m = 0;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec;
-       i += (long long)gridDim.x * blockDim.x) {
-    const uint4 v = x[i];
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t lo = w[j] & 0x7FFFu, hi = (w[j] >> 16) & 0x7FFFu;
-      // skip NaN patterns (exponent all ones, mantissa non-zero); infinities pass through
-      m = max(m, (lo > 0x7F80u) ? 0u : lo);
-      m = max(m, (hi > 0x7F80u) ? 0u : hi);
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  // one atomic per CTA: thousands of atomics on one address would serialise in the L2
-  __shared__ uint32_t warp_max[32];
-  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    m = threadIdx.x < (blockDim.x + 31) / 32 ? warp_max[threadIdx.x] : 0u;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    if (threadIdx.x == 0 && m) atomicMax(amax_bits, m);
-  }
-}
-
 // Round a non-negative finite float to the nearest E4M3 code (ties to even mantissa),
 // saturating at `max_code`.
 __device__ __forceinline__ uint32_t round_to_e4m3(float t, uint32_t max_code) {
@@ -61,70 +31,129 @@ __device__ __forceinline__ uint32_t round_to_fp4_idx(float a) {
          (uint32_t)(a >= 1.75f) + (uint32_t)(a > 2.5f) + (uint32_t)(a >= 3.5f) + (uint32_t)(a > 5.0f);
 }
 
-// One thread per 16-element block.
-__global__ void quant_act_kernel(const uint4* __restrict__ x, long long n_blocks, float sv_mag,
-                                 const float* __restrict__ scale_in, const uint32_t* __restrict__ amax_bits,
-                                 uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                                 float* __restrict__ scale_out) {
+// Quantize one 16-element block (Eq. 2-3, 6-7 with the candidates +sv and -sv): eight code bytes and the scale byte.
+__device__ __forceinline__ void quant_act_block(const uint4 v0, const uint4 v1, float d32, float d32x6, float sv_mag,
+                                                uint32_t& w0, uint32_t& w1, uint32_t& sbyte) {
+  const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+  float xv[16];
+  float bmax = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    xv[2 * j] = __uint_as_float(w[j] << 16);
+    xv[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    bmax = fmaxf(bmax, fmaxf(fabsf(xv[2 * j]), fabsf(xv[2 * j + 1])));
+  }
+  w0 = 0, w1 = 0, sbyte = 0;
+  if (bmax > 0.0f) {
+    const float tq = __fdiv_rn(bmax, d32x6);                         // Eq. 2 argument
+    uint32_t scode = round_to_e4m3(tq, 126u);
+    if (scode == 0) scode = 1;                                       // keep a non-empty block alive
+    const float denom = __fmul_rn(d32, scale_value(scode));
+    float e_pos = 0.0f, e_neg = 0.0f;
+    uint32_t std_code[16];
+    uint32_t take_pos = 0, take_neg = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float xs = __fdiv_rn(xv[j], denom);                      // the scaled block of Eq. 6
+      const uint32_t idx = round_to_fp4_idx(fabsf(xs));
+      const uint32_t neg = __float_as_uint(xs) >> 31;
+      const float r = neg ? -fp4_mag(idx) : fp4_mag(idx);
+      const float d_r = fabsf(__fsub_rn(xs, r));
+      const float d_p = fabsf(__fsub_rn(xs, sv_mag));
+      const float d_n = fabsf(__fsub_rn(xs, -sv_mag));
+      const bool tp = d_p < d_r, tn = d_n < d_r;                     // strictly closer only
+      const float qp = tp ? sv_mag : r, qn = tn ? -sv_mag : r;
+      const float dp = __fsub_rn(qp, xs), dn = __fsub_rn(qn, xs);
+      e_pos = __fadd_rn(e_pos, __fmul_rn(dp, dp));                   // ascending j, no fusion
+      e_neg = __fadd_rn(e_neg, __fmul_rn(dn, dn));
+      take_pos |= (uint32_t)tp << j;
+      take_neg |= (uint32_t)tn << j;
+      std_code[j] = idx ? (idx | (neg << 3)) : 0u;                   // a true zero is always code 0
+    }
+    const bool use_neg = e_neg < e_pos;                              // ties keep metadata 0 (+sv)
+    const uint32_t take = use_neg ? take_neg : take_pos;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint32_t c = ((take >> j) & 1u) ? 8u : std_code[j];
+      if (j < 8) w0 |= c << (4 * j); else w1 |= c << (4 * (j - 8));
+    }
+    sbyte = (use_neg ? 0x80u : 0u) | scode;
+  }
+}
+
+// One launch for the whole of razer_quant_act, one thread per 16-element block.  When the tensor scale has to be
+// computed (Eq. 1), the grid first takes the tensor maximum: every CTA folds its share into sync[0] and counts
+// itself in sync[1], and all of them meet there (the launch is cooperative, so every CTA is resident; the wait is
+// bounded all the same).  sync[] must be zero when the kernel starts; the last CTA to finish sets it back to zero.
+__global__ void __launch_bounds__(256) quant_act_fused_kernel(const uint4* __restrict__ x, long long n_blocks, float sv_mag,
+                                                             const float* __restrict__ scale_in, uint32_t* sync,
+                                                             uint2* __restrict__ codes, uint8_t* __restrict__ scales,
+                                                             float* __restrict__ scale_out) {
+  __shared__ uint32_t warp_max[8];
+  __shared__ uint32_t amax_shared;
   float d32;
   if (scale_in) {
     d32 = *scale_in;
   } else {
-    const float amax = __uint_as_float(*amax_bits << 16);
+    uint32_t m = 0;
+    const long long n_vec = n_blocks * 2;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (long long)gridDim.x * blockDim.x) {
+      const uint4 v = x[i];
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t lo = w[j] & 0x7FFFu, hi = (w[j] >> 16) & 0x7FFFu;
+        m = max(m, (lo > 0x7F80u) ? 0u : lo);                          // NaN patterns are skipped
+        m = max(m, (hi > 0x7F80u) ? 0u : hi);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int i = 1; i < 8; ++i) m = max(m, warp_max[i]);
+      if (m) atomicMax(&sync[0], m);
+      __threadfence();
+      atomicAdd(&sync[1], 1u);
+      // all CTAs are resident (cooperative launch); the bound only guards against a dirty sync[]
+      uint32_t seen = 0;
+      for (uint32_t spins = 0; spins < (1u << 22); ++spins) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(sync + 1) : "memory");
+        if (seen >= gridDim.x) break;
+        __nanosleep(64);
+      }
+      uint32_t a;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(a) : "l"(sync) : "memory");
+      amax_shared = seen >= gridDim.x ? a : 0xFFFFFFFFu;               // gave up: flagged below with a NaN scale
+    }
+    __syncthreads();
+    const uint32_t bits = amax_shared;
+    if (bits == 0xFFFFFFFFu) {
+      if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = __uint_as_float(0x7FC00000u);
+      return;
+    }
+    const float amax = __uint_as_float(bits << 16);
     d32 = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, __fmul_rn(448.0f, 6.0f));   // Eq. 1
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = d32;
   const float d32x6 = __fmul_rn(d32, 6.0f);
   for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_blocks;
        t += (long long)gridDim.x * blockDim.x) {
-    const uint4 v0 = x[2 * t], v1 = x[2 * t + 1];
-    const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    float xv[16];
-    float bmax = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      xv[2 * j] = __uint_as_float(w[j] << 16);
-      xv[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-      bmax = fmaxf(bmax, fmaxf(fabsf(xv[2 * j]), fabsf(xv[2 * j + 1])));
-    }
-    uint32_t w0 = 0, w1 = 0, sbyte = 0;
-    if (bmax > 0.0f) {
-      const float tq = __fdiv_rn(bmax, d32x6);                         // Eq. 2 argument
-      uint32_t scode = round_to_e4m3(tq, 126u);
-      if (scode == 0) scode = 1;                                       // keep a non-empty block alive
-      const float denom = __fmul_rn(d32, scale_value(scode));
-      float e_pos = 0.0f, e_neg = 0.0f;
-      uint32_t std_code[16];
-      uint32_t take_pos = 0, take_neg = 0;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float xs = __fdiv_rn(xv[j], denom);                      // the scaled block of Eq. 6
-        const uint32_t idx = round_to_fp4_idx(fabsf(xs));
-        const uint32_t neg = __float_as_uint(xs) >> 31;
-        const float r = neg ? -fp4_mag(idx) : fp4_mag(idx);
-        const float d_r = fabsf(__fsub_rn(xs, r));
-        const float d_p = fabsf(__fsub_rn(xs, sv_mag));
-        const float d_n = fabsf(__fsub_rn(xs, -sv_mag));
-        const bool tp = d_p < d_r, tn = d_n < d_r;                     // strictly closer only
-        const float qp = tp ? sv_mag : r, qn = tn ? -sv_mag : r;
-        const float dp = __fsub_rn(qp, xs), dn = __fsub_rn(qn, xs);
-        e_pos = __fadd_rn(e_pos, __fmul_rn(dp, dp));                   // ascending j, no fusion
-        e_neg = __fadd_rn(e_neg, __fmul_rn(dn, dn));
-        take_pos |= (uint32_t)tp << j;
-        take_neg |= (uint32_t)tn << j;
-        std_code[j] = idx ? (idx | (neg << 3)) : 0u;                   // a true zero is always code 0
-      }
-      const bool use_neg = e_neg < e_pos;                              // ties keep metadata 0 (+sv)
-      const uint32_t take = use_neg ? take_neg : take_pos;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const uint32_t c = ((take >> j) & 1u) ? 8u : std_code[j];
-        if (j < 8) w0 |= c << (4 * j); else w1 |= c << (4 * (j - 8));
-      }
-      sbyte = (use_neg ? 0x80u : 0u) | scode;
-    }
+    uint32_t w0, w1, sbyte;
+    quant_act_block(x[2 * t], x[2 * t + 1], d32, d32x6, sv_mag, w0, w1, sbyte);
     codes[t] = make_uint2(w0, w1);
     scales[t] = (uint8_t)sbyte;
+  }
+  if (!scale_in) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const uint32_t prev = atomicAdd(&sync[1], 1u);
+      if (prev + 1 == 2 * gridDim.x) {                                 // everyone has read the maximum: leave sync[] clean
+        sync[0] = 0;
+        sync[1] = 0;
+      }
+    }
   }
 }
 
@@ -251,29 +280,34 @@ int launch_quant_weight(const float* w, int N, int K, float m0, float m1, int re
 }
 
 int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* scale_in,
-                     uint32_t* amax_scratch, uint8_t* codes, uint8_t* scales, float* scale_out,
+                     uint32_t* sync_scratch, uint8_t* codes, uint8_t* scales, float* scale_out,
                      cudaStream_t st) {
   const long long n_blocks = (long long)M * (K / 16);
-  const long long n_vec = n_blocks * 2;
   const int threads = 256;
-  auto grid = [&](long long n) {
-    long long b = (n + threads - 1) / threads;
-    return (int)(b < 1 ? 1 : (b > 148LL * 16 ? 148LL * 16 : b));
-  };
-  if (!scale_in) {
-    RAZER_TRY(check_cuda(cudaMemsetAsync(amax_scratch, 0, sizeof(uint32_t), st), "amax memset"));
-    {
-      long long b = (n_vec + threads * 4 - 1) / (threads * 4);        // four vectors per thread, at most two CTAs per SM
-      const int g2 = (int)(b < 1 ? 1 : (b > 296 ? 296 : b));
-      act_amax_kernel<<<g2, threads, 0, st>>>((const uint4*)x, n_vec, amax_scratch);
-    }
-    count_launches(1);
-    RAZER_TRY(check_cuda(cudaGetLastError(), "act_amax_kernel launch"));
+  static int max_ctas = 0;                                             // CTAs that are resident together (cooperative launch)
+  if (!max_ctas) {
+    int dev = 0, sms = 0, per_sm = 0;
+    RAZER_TRY(check_cuda(cudaGetDevice(&dev), "cudaGetDevice"));
+    RAZER_TRY(check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"));
+    RAZER_TRY(check_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_act_fused_kernel, threads, 0),
+                         "cudaOccupancyMaxActiveBlocksPerMultiprocessor"));
+    max_ctas = sms * (per_sm < 1 ? 1 : per_sm);
   }
-  quant_act_kernel<<<grid(n_blocks), threads, 0, st>>>((const uint4*)x, n_blocks, sv_mag, scale_in,
-                                                       amax_scratch, (uint2*)codes, scales, scale_out);
+  long long b = (n_blocks + threads - 1) / threads;
+  const int grid = (int)(b < 1 ? 1 : (b > max_ctas ? max_ctas : b));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(threads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = scale_in ? 0 : 1;                                     // the grid only meets when it computes the scale
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_fused_kernel, (const uint4*)x, n_blocks, sv_mag, scale_in,
+                                           sync_scratch, (uint2*)codes, scales, scale_out);
   count_launches(1);
-  return check_cuda(cudaGetLastError(), "quant_act_kernel launch");
+  return check_cuda(e, "quant_act_fused_kernel launch");
 }
 
 }  // namespace razer
