@@ -55,7 +55,8 @@ enum { RAZER_OP_GEMV = 0, RAZER_OP_GEMM = 1, RAZER_OP_GEMM_W4A4 = 2 };
 typedef struct razer_desc {
   int32_t N;            /* rows (output features), >= 1                                     */
   int32_t K;            /* columns (reduction dim), multiple of 16                          */
-  int32_t block;        /* elements per block; must be 16 (Sec. 3)                          */
+  int32_t block;        /* elements per scale block along K: 16 (Sec. 3) or 32, 64, 128
+                           (the block-size study of Sec. 5); K must be a multiple of it      */
   int32_t scale_fmt;    /* RAZER_SCALE_E3M3_META2 for weights                                */
   int32_t remap_code;   /* which zero nibble is the special value in the interchange codes:
                            0x8 (negative zero, default) or 0x0                               */
@@ -75,7 +76,8 @@ int razer_version(void);
 unsigned long long razer_kernel_launches(void);
 
 /* Size in bytes of the GPU-internal packed form of the tensor `d` describes.
- * The packed form has the same 4.5 bits per weight (codes + scale bytes), padded to whole
+ * The packed form has 4.5 bits per weight (codes + one scale byte per 16 elements: the byte
+ * of a larger block is repeated, so that every kernel reads one layout), padded to whole
  * 128-row x 64-column tiles. */
 int razer_packed_bytes(const razer_desc* d, size_t* bytes_out);
 
@@ -176,15 +178,23 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag,
                     float* tensor_scale_out_dev, void* stream);
 
 /* Weight quantizer on the GPU (Sec. 4.2, Eq. 1-3 and 6-7 with the 6-bit E3M3 block scale of
- * Sec. 4.1): every block of 16 along K is quantized once per allowed special value, in
- * metadata order +sv_mag[0], +sv_mag[1], -sv_mag[0], -sv_mag[1], and the lowest squared
- * error wins (ties: the smaller metadata value).  w_dev: FP32 [N][K], K multiple of 16,
- * 16-byte aligned.  tensor_scale_in_dev / amax_scratch_dev as in razer_quant_act.  Writes
- * the interchange format that razer_pack_layout reads: codes_dev [N][K/2], scales_dev
- * [N][K/16] ([meta(2) | E3M3 code(6)]), special value = remap_code (0x8 or 0x0), and the
- * tensor scale to tensor_scale_out_dev.  Every FP32 step is a single IEEE operation in a
- * fixed order, so the result is reproducible bit for bit.  Asynchronous on `stream`. */
-int razer_quant_weight(const float* w_dev, int N, int K, const float sv_mag[2], int remap_code,
+ * Sec. 4.1): every block along K is quantized once per allowed special value, in metadata
+ * order +sv_mag[0], +sv_mag[1], -sv_mag[0], -sv_mag[1], and the lowest squared error wins
+ * (ties: the smaller metadata value).  `block` = elements per scale block along K (16, 32, 64
+ * or 128).  scale_aware = 0: all four share the scale of Eq. 2 (block maximum -> 6), as the
+ * equations are printed.  scale_aware != 0: a special value beyond 6 whose sign is that of the
+ * block's first largest element also competes with a scale of its own (block maximum -> its
+ * magnitude); the errors are then compared in the tensor's units and the standard four come
+ * first in a tie.  The output format is the same either way.
+ * w_dev: FP32 [N][K], K a multiple of `block`, 16-byte aligned.  tensor_scale_in_dev as in
+ * razer_quant_act; amax_scratch_dev: one device uint32 (needed when the scale is computed; the
+ * call clears it itself).  Writes the interchange format that razer_pack_layout reads:
+ * codes_dev [N][K/2], scales_dev [N][K/block] ([meta(2) | E3M3 code(6)]), special value =
+ * remap_code (0x8 or 0x0), and the tensor scale to tensor_scale_out_dev.  Every FP32 step is a
+ * single IEEE operation in a fixed order, so the result is reproducible bit for bit.
+ * Asynchronous on `stream`. */
+int razer_quant_weight(const float* w_dev, int N, int K, int block, int scale_aware,
+                       const float sv_mag[2], int remap_code,
                        const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev,
                        uint8_t* codes_dev, uint8_t* scales_dev, float* tensor_scale_out_dev,
                        void* stream);

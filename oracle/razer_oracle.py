@@ -14,6 +14,7 @@ What is here, with the passage each function follows:
   round_to_fp4         Eq. 3's rounding onto the FP4 set
   offset_decoder_sv    Sec. 4.4 (offset-register special-value decoder)
   quantize             Eq. 1-3 + Eq. 6-7 (tensor scale, block scale, special-value argmin)
+  quantize_scale_aware Eq. 6-7 with the block scale of Eq. 2 chosen together with the special value
   decode_block_values  Sec. 4.2 + Sec. 4.4 (code -> value with the remapped zero)
   dequant_d1/_d2       the dequantization product Delta32 * Delta8 * Xbar (Sec. 3)
   matmul_w4a16/_w4a4   definition: FP64-accumulated product rounded once to bf16
@@ -286,6 +287,99 @@ def quantize(x: np.ndarray, scale_fmt: int = SCALE_E3M3_META2, sv_mag=(5.0, 8.0)
         dbg = dict(xs=xs, errs32=errs32, errs64=errs64, err_fp4=np.sum(d0 * d0, axis=2),
                    meta=meta, scode=scode, near_tie=_near_ties(errs64))
         return packed, sbyte, d32, dbg
+    return packed, sbyte, d32
+
+
+def quantize_scale_aware(x: np.ndarray, scale_fmt: int = SCALE_E3M3_META2, sv_mag=(5.0, 8.0),
+                         remap_code: int = 0x8, block: int = BLOCK, tensor_scale=None,
+                         return_debug: bool = False):
+    """Eq. 6-7 with the block scale chosen together with the special value.
+
+    Eq. 2 scales a block so that its largest magnitude lands on Qmax = 6, whatever v is
+    (Eq. 1-2 do not mention v), so a special value beyond 6 can only be reached where the
+    scale clamps.  Here a special value v with |v| > 6 whose sign is that of the block's
+    largest element also brings a scale of its own: Eq. 2 with Qmax replaced by |v|, the
+    largest magnitude of Q + {v} on that side.  Candidates, in this order:
+      0..n-1  the special values in metadata order with the scale of Eq. 2 (as `quantize`)
+      n..     for every such v (metadata order) the pair (v, scale of Eq. 2 with Qmax = |v|)
+    Each candidate's scaled-domain error e = sum_j (q_j - xs_j)^2 is formed exactly as in
+    `quantize` (FP32, ascending j) and compared in the tensor's own units as
+    fl32(fl32(d * d) * e) with d = fl32(D32 * s) the candidate's dequantization step; the
+    first minimum wins.  D32 stays Eq. 1's.  The output format is unchanged (codes, scale
+    byte = metadata | scale code), so every decoder reads it as it stands.
+    """
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    assert x.ndim == 2 and x.shape[1] % block == 0 and remap_code in (0x0, 0x8)
+    R, C = x.shape
+    nb = C // block
+    f32 = np.float32
+    grid = scale_grid(scale_fmt)
+    cands = sv_candidates(sv_mag, scale_fmt)
+    shift = 8 - meta_bits(scale_fmt)
+    if tensor_scale is None:
+        amax = f32(np.max(np.abs(x))) if x.size else f32(0)
+        d32 = f32(1.0) if amax == 0 else f32(amax / f32(f32(grid[-1]) * f32(6.0)))
+    else:
+        d32 = f32(tensor_scale)
+    xb = x.reshape(R, nb, block)
+    absx = np.abs(xb)
+    bmax = np.max(absx, axis=2).astype(np.float32)
+    top = np.take_along_axis(xb, np.argmax(absx, axis=2)[:, :, None], axis=2)[:, :, 0]   # first largest element
+    top_neg = np.signbit(top)
+
+    def scale_for(qmax):
+        t = (bmax / f32(d32 * f32(qmax))).astype(np.float32)
+        sc = round_to_scale(t, scale_fmt)
+        sc = np.where((bmax > 0) & (sc == 0), 1, sc)
+        return np.where(bmax == 0, 0, sc).astype(np.uint8)
+
+    def evaluate(v, scode):
+        sval = grid[scode].astype(np.float32)
+        denom = (d32 * sval).astype(np.float32)
+        safe = np.where(denom == 0, f32(1.0), denom)
+        xs = (xb / safe[:, :, None]).astype(np.float32)
+        xs = np.where(denom[:, :, None] == 0, f32(0.0), xs)
+        ridx = round_to_fp4(xs)
+        rval = (np.where(np.signbit(xs), -1.0, 1.0) * _FP4_MAGS[ridx]).astype(np.float32)
+        take = np.abs(xs - f32(v)).astype(np.float32) < np.abs(xs - rval).astype(np.float32)
+        q = np.where(take, f32(v), rval).astype(np.float32)
+        diff = (q - xs).astype(np.float32)
+        sq = (diff * diff).astype(np.float32)
+        acc = np.zeros((R, nb), dtype=np.float32)
+        for j in range(block):
+            acc = (acc + sq[:, :, j]).astype(np.float32)
+        err32 = ((denom * denom).astype(np.float32) * acc).astype(np.float32)
+        d64 = (q.astype(np.float64) - xs.astype(np.float64)) * denom.astype(np.float64)[:, :, None]
+        other_zero = remap_code ^ 0x8
+        std = (ridx | (np.signbit(xs).astype(np.uint8) << 3)).astype(np.uint8)
+        std = np.where(ridx == 0, other_zero, std).astype(np.uint8)
+        code = np.where(take, np.uint8(remap_code), std).astype(np.uint8)
+        code = np.where((scode == 0)[:, :, None], np.uint8(other_zero), code)
+        return err32, np.sum(d64 * d64, axis=2), code
+
+    s6 = scale_for(6.0)
+    options = [(ci, v, s6, np.ones((R, nb), dtype=bool)) for ci, v in enumerate(cands)]
+    for ci, v in enumerate(cands):
+        if abs(v) > 6.0:
+            options.append((ci, v, scale_for(abs(v)), (top_neg == (v < 0)) & (bmax > 0)))
+    errs32 = np.empty((len(options), R, nb), dtype=np.float32)
+    errs64 = np.empty((len(options), R, nb), dtype=np.float64)
+    codes_all = np.empty((len(options), R, nb, block), dtype=np.uint8)
+    for oi, (ci, v, sc, ok) in enumerate(options):
+        e32, e64, code = evaluate(v, sc)
+        errs32[oi] = np.where(ok, e32, np.float32(np.inf))
+        errs64[oi] = np.where(ok, e64, np.inf)
+        codes_all[oi] = code
+    pick = np.argmin(errs32, axis=0)                                     # first minimum
+    code = np.take_along_axis(codes_all, pick[None, :, :, None], axis=0)[0].reshape(R, C)
+    meta = np.array([o[0] for o in options], dtype=np.uint8)[pick]
+    scode = np.take_along_axis(np.stack([o[2] for o in options]), pick[None], axis=0)[0]
+    packed = (code[:, 0::2] | (code[:, 1::2] << 4)).astype(np.uint8)
+    sbyte = ((meta.astype(np.uint16) << shift) | scode).astype(np.uint8)
+    sbyte = np.where(scode == 0, 0, sbyte).astype(np.uint8)
+    if return_debug:
+        return packed, sbyte, d32, dict(errs32=errs32, errs64=errs64, pick=pick, n_standard=len(cands),
+                                        near_tie=_near_ties(np.where(np.isfinite(errs64), errs64, 1e300)))
     return packed, sbyte, d32
 
 

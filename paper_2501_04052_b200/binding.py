@@ -61,7 +61,7 @@ _lib.razer_gemv_host.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, 
 _lib.razer_gemv_static.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_int, c_void_p, c_void_p]
 _lib.razer_quant_act.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p, c_void_p,
                                  c_void_p, c_void_p]
-_lib.razer_quant_weight.argtypes = [c_void_p, c_int, c_int, POINTER(c_float), c_int, c_void_p, c_void_p, c_void_p,
+_lib.razer_quant_weight.argtypes = [c_void_p, c_int, c_int, c_int, c_int, POINTER(c_float), c_int, c_void_p, c_void_p, c_void_p,
                                     c_void_p, c_void_p, c_void_p]
 _lib.razer_decode_act.argtypes = [c_void_p, c_void_p, c_int, c_int, c_float, c_void_p, c_void_p]
 _lib.razer_gemm_w4a4.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_int,
@@ -216,17 +216,17 @@ def razer_quant_act(x: torch.Tensor, sv_mag: float = 5.0, tensor_scale: torch.Te
 
 
 def razer_quant_weight(w: torch.Tensor, sv_mag=(5.0, 8.0), remap_code: int = 0x8,
-                       tensor_scale: torch.Tensor | None = None):
-    """w FP32 [N, K] (device) -> (codes uint8 [N, K/2], scales uint8 [N, K/16], tensor scale float32 [1]) in the
+                       tensor_scale: torch.Tensor | None = None, block: int = 16, scale_aware: bool = False):
+    """w FP32 [N, K] (device) -> (codes uint8 [N, K/2], scales uint8 [N, K/block], tensor scale float32 [1]) in the
     interchange format that razer_pack_layout reads."""
     assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
     N, K = w.shape
     codes = torch.empty((N, K // 2), dtype=torch.uint8, device=w.device)
-    scales = torch.empty((N, K // 16), dtype=torch.uint8, device=w.device)
+    scales = torch.empty((N, K // block), dtype=torch.uint8, device=w.device)
     out_scale = torch.empty(1, dtype=torch.float32, device=w.device)
     scratch = torch.empty(1, dtype=torch.int32, device=w.device)
     mags = (c_float * 2)(float(sv_mag[0]), float(sv_mag[1]))
-    _check(_lib.razer_quant_weight(_ptr(w), N, K, mags, int(remap_code), _ptr(tensor_scale), _ptr(scratch),
+    _check(_lib.razer_quant_weight(_ptr(w), N, K, int(block), int(bool(scale_aware)), mags, int(remap_code), _ptr(tensor_scale), _ptr(scratch),
                                    _ptr(codes), _ptr(scales), _ptr(out_scale), _stream()))
     return codes, scales, out_scale
 

@@ -40,7 +40,9 @@ int check_desc(const razer_desc* d) {
   if (!d) return set_error(RAZER_ERR_INVALID_ARG, "descriptor is NULL");
   if (d->N < 1 || d->K < 16) return set_error(RAZER_ERR_INVALID_ARG, "N=%d K=%d out of range", d->N, d->K);
   if (d->K % 16) return set_error(RAZER_ERR_INVALID_ARG, "K=%d is not a multiple of 16", d->K);
-  if (d->block != 16) return set_error(RAZER_ERR_UNSUPPORTED, "block size %d (only 16 is built)", d->block);
+  if (d->block != 16 && d->block != 32 && d->block != 64 && d->block != 128)
+    return set_error(RAZER_ERR_UNSUPPORTED, "block size %d (16, 32, 64 and 128 are built)", d->block);
+  if (d->K % d->block) return set_error(RAZER_ERR_INVALID_ARG, "K=%d is not a multiple of the block size %d", d->K, d->block);
   if (d->scale_fmt != RAZER_SCALE_E3M3_META2)
     return set_error(RAZER_ERR_UNSUPPORTED, "weight scale format %d (only E3M3 + 2 metadata bits)", d->scale_fmt);
   if (d->remap_code != 0x8 && d->remap_code != 0x0)
@@ -64,8 +66,8 @@ static int check_ptr(const void* p, size_t align, const char* name) {
 int launch_pack(const razer_desc*, const uint8_t*, const uint8_t*, void*, cudaStream_t);
 int launch_dequant(const razer_desc*, const void*, void*, int, cudaStream_t);
 int launch_decode_act(const uint8_t*, const uint8_t*, int, int, float, void*, cudaStream_t);
-int launch_quant_weight(const float*, int, int, float, float, int, const float*, uint32_t*, uint8_t*, uint8_t*,
-                        float*, cudaStream_t);
+int launch_quant_weight(const float*, int, int, int, int, float, float, int, const float*, uint32_t*, uint8_t*,
+                        uint8_t*, float*, cudaStream_t);
 int launch_quant_act(const void*, int, int, float, const float*, uint32_t*, uint8_t*, uint8_t*, float*,
                      cudaStream_t);
 int launch_gemv_simt(const razer_desc*, const void*, const void*, int, const float*, void*, void*, size_t,
@@ -263,10 +265,13 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag, const float* 
                           act_scales_dev, tensor_scale_out_dev, (cudaStream_t)stream);
 }
 
-int razer_quant_weight(const float* w_dev, int N, int K, const float sv_mag[2], int remap_code,
+int razer_quant_weight(const float* w_dev, int N, int K, int block, int scale_aware, const float sv_mag[2], int remap_code,
                        const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev, uint8_t* codes_dev,
                        uint8_t* scales_dev, float* tensor_scale_out_dev, void* stream) {
-  if (N < 1 || K < 16 || K % 16) return set_error(RAZER_ERR_INVALID_ARG, "N=%d K=%d invalid (K %% 16 == 0)", N, K);
+  if (block != 16 && block != 32 && block != 64 && block != 128)
+    return set_error(RAZER_ERR_UNSUPPORTED, "block size %d (16, 32, 64 and 128 are built)", block);
+  if (N < 1 || K < block || K % block)
+    return set_error(RAZER_ERR_INVALID_ARG, "N=%d K=%d invalid (K must be a multiple of the block size %d)", N, K, block);
   if (!sv_mag) return set_error(RAZER_ERR_INVALID_ARG, "sv_mag is NULL");
   if (remap_code != 0x8 && remap_code != 0x0)
     return set_error(RAZER_ERR_INVALID_ARG, "remap_code 0x%x is not a zero code", remap_code);
@@ -278,7 +283,7 @@ int razer_quant_weight(const float* w_dev, int N, int K, const float sv_mag[2], 
   RAZER_TRY(check_ptr(scales_dev, 1, "scales_dev"));
   RAZER_TRY(check_ptr(tensor_scale_out_dev, 4, "tensor_scale_out_dev"));
   if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 4, "amax_scratch_dev"));
-  return launch_quant_weight(w_dev, N, K, sv_mag[0], sv_mag[1], remap_code, tensor_scale_in_dev, amax_scratch_dev,
+  return launch_quant_weight(w_dev, N, K, block, scale_aware != 0, sv_mag[0], sv_mag[1], remap_code, tensor_scale_in_dev, amax_scratch_dev,
                              codes_dev, scales_dev, tensor_scale_out_dev, (cudaStream_t)stream);
 }
 

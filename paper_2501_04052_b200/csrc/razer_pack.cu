@@ -5,8 +5,10 @@ namespace razer {
 
 // One thread per (row tile, k chunk, block, row): reads the interchange-format block
 // (8 code bytes + 1 scale byte), canonicalises it and writes it at its packed position.
+// `sub` = 16-element groups per scale block (block size / 16): the packed form always carries one scale byte per 16
+// elements, so a larger block's byte is repeated for each of its groups and the kernels need not know the block size.
 __global__ void pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
-                            uint8_t* __restrict__ packed, Geometry g, int remap_code) {
+                            uint8_t* __restrict__ packed, Geometry g, int remap_code, int sub) {
   const long long total = (long long)g.row_tiles * g.k_chunks * CHUNK_BLOCKS * TILE_ROWS;
   for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (long long)gridDim.x * blockDim.x) {
@@ -22,7 +24,7 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __
       const uint2 c = *reinterpret_cast<const uint2*>(codes + (size_t)n * (g.K / 2) + (size_t)kb * 8);
       w0 = c.x;
       w1 = c.y;
-      sb = scales[(size_t)n * (g.K / 16) + kb];
+      sb = scales[(size_t)n * (g.K / 16 / sub) + kb / sub];
     }
     // bit 3 of each nibble of nz is set iff the nibble's magnitude (low three bits) is non-zero
     auto canon = [&](uint32_t w, bool negate) -> uint32_t {
@@ -140,7 +142,7 @@ int launch_pack(const razer_desc* d, const uint8_t* codes, const uint8_t* scales
                 cudaStream_t st) {
   const Geometry g = make_geometry(d->N, d->K);
   const long long total = (long long)g.row_tiles * g.k_chunks * CHUNK_BLOCKS * TILE_ROWS;
-  pack_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, scales, (uint8_t*)packed, g, d->remap_code);
+  pack_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, scales, (uint8_t*)packed, g, d->remap_code, d->block / 16);
   count_launches(1);
   RAZER_TRY(check_cuda(cudaGetLastError(), "pack_kernel launch"));
   pack_done_kernel<<<1, 32, 0, st>>>();

@@ -186,11 +186,20 @@ __global__ void weight_amax_kernel(const float4* __restrict__ w, long long n_vec
   }
 }
 
-// One thread per 16-element block.
-__global__ void quant_weight_kernel(const float4* __restrict__ w, long long n_blocks, float m0, float m1,
+// One thread per scale block of `sub` groups of 16 elements (block size 16 * sub).  Three walks over the block:
+// its maximum, the candidates' errors (FP32, ascending element order across the whole block), and the codes
+// under the winning candidate.
+//
+// AWARE = false: the four special values share the scale of Eq. 2 (block maximum -> 6), Eq. 6-7 as printed.
+// AWARE = true: a special value beyond 6 whose sign is that of the block's first largest element brings a
+// second candidate with a scale of its own (block maximum -> |v|); slots 4 and 5 hold those for m0 and m1.
+// Errors are then compared in the tensor's units, fl32(fl32(d * d) * e) with d the candidate's step.
+template <bool AWARE>
+__global__ void quant_weight_kernel(const float4* __restrict__ w, long long n_blocks, int sub, float m0, float m1,
                                     uint32_t remap_code, const float* __restrict__ scale_in,
                                     const uint32_t* __restrict__ amax_bits, uint2* __restrict__ codes,
                                     uint8_t* __restrict__ scales, float* __restrict__ scale_out) {
+  constexpr int NC = AWARE ? 6 : 4;
   float d32;
   if (scale_in) {
     d32 = *scale_in;
@@ -199,69 +208,106 @@ __global__ void quant_weight_kernel(const float4* __restrict__ w, long long n_bl
     d32 = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, __fmul_rn(1.875f, 6.0f));   // Eq. 1
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = d32;
-  const float d32x6 = __fmul_rn(d32, 6.0f);
   const uint32_t other_zero = remap_code ^ 8u;
-  const float cand[4] = {m0, m1, -m0, -m1};
+  const float mags[2] = {m0, m1};
   for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_blocks;
        t += (long long)gridDim.x * blockDim.x) {
-    float xv[16];
+    const float4* src = w + 4 * t * sub;
     float bmax = 0.0f;
+    uint32_t top_neg = 0;                                              // sign of the first largest element
+    for (int q = 0; q < 4 * sub; ++q) {
+      const float4 v = src[q];
+      const float xv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float4 v = w[4 * t + q];
-      xv[4 * q] = v.x, xv[4 * q + 1] = v.y, xv[4 * q + 2] = v.z, xv[4 * q + 3] = v.w;
-      bmax = fmaxf(bmax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+      for (int j = 0; j < 4; ++j)
+        if (fabsf(xv[j]) > bmax) { bmax = fabsf(xv[j]); top_neg = __float_as_uint(xv[j]) >> 31; }
     }
-    uint32_t w0 = other_zero * 0x11111111u, w1 = w0, sbyte = 0;
+    uint32_t sbyte = 0;
+    float denom = 1.0f, sv = m0;
     if (bmax > 0.0f) {
-      const float tq = __fdiv_rn(bmax, d32x6);                         // Eq. 2 argument
-      uint32_t scode = round_to_e4m3(tq, 63u);
-      if (scode == 0) scode = 1;                                       // keep a non-empty block alive
-      const float denom = __fmul_rn(d32, scale_value(scode));
-      float err[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      uint32_t take[4] = {0, 0, 0, 0};
-      uint32_t std_lo = 0, std_hi = 0;                                 // plain FP4 codes, eight nibbles each
+      float cv[NC], cd[NC];
+      uint32_t cs[NC], cm[NC];
+      bool ok[NC];
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float xs = __fdiv_rn(xv[j], denom);                      // the scaled block of Eq. 6
-        const uint32_t idx = round_to_fp4_idx(fabsf(xs));
-        const uint32_t neg = __float_as_uint(xs) >> 31;
-        const float r = neg ? -fp4_mag(idx) : fp4_mag(idx);
-        const float d_r = fabsf(__fsub_rn(xs, r));
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const bool tk = fabsf(__fsub_rn(xs, cand[c])) < d_r;         // strictly closer only
-          const float d = __fsub_rn(tk ? cand[c] : r, xs);
-          err[c] = __fadd_rn(err[c], __fmul_rn(d, d));                 // ascending j, no fusion
-          take[c] |= (uint32_t)tk << j;
-        }
-        const uint32_t sc = idx ? (idx | (neg << 3)) : other_zero;     // a true zero is always the other zero code
-        if (j < 8) std_lo |= sc << (4 * j); else std_hi |= sc << (4 * (j - 8));
+      for (int c = 0; c < NC; ++c) {
+        const float qmax = c < 4 ? 6.0f : mags[c - 4];
+        const float tq = __fdiv_rn(bmax, __fmul_rn(d32, qmax));        // Eq. 2 argument
+        uint32_t scode = round_to_e4m3(tq, 63u);
+        if (scode == 0) scode = 1;                                     // keep a non-empty block alive
+        cs[c] = scode;
+        cd[c] = __fmul_rn(d32, scale_value(scode));
+        cm[c] = c < 4 ? (uint32_t)c : (top_neg * 2u + (uint32_t)(c - 4));
+        cv[c] = (cm[c] & 2u) ? -mags[cm[c] & 1u] : mags[cm[c] & 1u];
+        ok[c] = c < 4 || mags[c - 4] > 6.0f;
       }
-      uint32_t meta = 0;                                               // first minimum: ties keep the smaller metadata
+      float err[NC];
+#pragma unroll
+      for (int c = 0; c < NC; ++c) err[c] = 0.0f;
+#pragma unroll 1
+      for (int q = 0; q < 4 * sub; ++q) {
+        const float4 v = src[q];
+        const float xv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int c = 0; c < NC; ++c) {
+            if (c >= 4 && !ok[c]) continue;
+            const float xs = __fdiv_rn(xv[j], cd[c]);                  // the scaled block of Eq. 6
+            const uint32_t idx = round_to_fp4_idx(fabsf(xs));
+            const float r = (__float_as_uint(xs) >> 31) ? -fp4_mag(idx) : fp4_mag(idx);
+            const bool tk = fabsf(__fsub_rn(xs, cv[c])) < fabsf(__fsub_rn(xs, r));   // strictly closer only
+            const float d = __fsub_rn(tk ? cv[c] : r, xs);
+            err[c] = __fadd_rn(err[c], __fmul_rn(d, d));               // ascending element order, no fusion
+          }
+        }
+      }
+      if (AWARE) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) err[c] = __fmul_rn(__fmul_rn(cd[c], cd[c]), err[c]);
+      }
+      int pick = 0;                                                    // first minimum: ties keep the earlier candidate
       float best = err[0];
 #pragma unroll
-      for (int c = 1; c < 4; ++c)
-        if (err[c] < best) { best = err[c]; meta = c; }
-      const uint32_t tk = take[0] * (meta == 0) | take[1] * (meta == 1) | take[2] * (meta == 2) | take[3] * (meta == 3);
-      w0 = std_lo, w1 = std_hi;
+      for (int c = 1; c < NC; ++c)
+        if (ok[c] && err[c] < best) { best = err[c]; pick = c; }
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if ((tk >> j) & 1u) {
-          if (j < 8) w0 = (w0 & ~(0xFu << (4 * j))) | (remap_code << (4 * j));
-          else w1 = (w1 & ~(0xFu << (4 * (j - 8)))) | (remap_code << (4 * (j - 8)));
-        }
-      sbyte = (meta << 6) | scode;
+      for (int c = 0; c < NC; ++c)
+        if (c == pick) { sbyte = (cm[c] << 6) | cs[c]; denom = cd[c]; sv = cv[c]; }
     }
-    codes[t] = make_uint2(w0, w1);
+#pragma unroll 1
+    for (int g = 0; g < sub; ++g) {
+      uint32_t wd[2] = {other_zero * 0x11111111u, other_zero * 0x11111111u};
+      if (bmax > 0.0f) {
+        wd[0] = wd[1] = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 v = src[4 * g + q];
+          const float xv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float xs = __fdiv_rn(xv[j], denom);
+            const uint32_t idx = round_to_fp4_idx(fabsf(xs));
+            const uint32_t neg = __float_as_uint(xs) >> 31;
+            const float r = neg ? -fp4_mag(idx) : fp4_mag(idx);
+            const bool tk = fabsf(__fsub_rn(xs, sv)) < fabsf(__fsub_rn(xs, r));
+            const uint32_t c = tk ? remap_code : (idx ? (idx | (neg << 3)) : other_zero);   // a true zero is always the other zero code
+            const int e = 4 * q + j;
+            wd[e >> 3] |= c << (4 * (e & 7));
+          }
+        }
+      }
+      codes[t * sub + g] = make_uint2(wd[0], wd[1]);
+    }
     scales[t] = (uint8_t)sbyte;
   }
 }
 
-int launch_quant_weight(const float* w, int N, int K, float m0, float m1, int remap_code, const float* scale_in,
+int launch_quant_weight(const float* w, int N, int K, int block, int scale_aware, float m0, float m1, int remap_code,
+                        const float* scale_in,
                         uint32_t* amax_scratch, uint8_t* codes, uint8_t* scales, float* scale_out, cudaStream_t st) {
-  const long long n_blocks = (long long)N * (K / 16);
-  const long long n_vec = n_blocks * 4;
+  const int sub = block / 16;
+  const long long n_blocks = (long long)N * (K / block);
+  const long long n_vec = (long long)N * (K / 4);
   const int threads = 256;
   if (!scale_in) {
     RAZER_TRY(check_cuda(cudaMemsetAsync(amax_scratch, 0, sizeof(uint32_t), st), "amax memset"));
@@ -273,8 +319,12 @@ int launch_quant_weight(const float* w, int N, int K, float m0, float m1, int re
   }
   long long b = (n_blocks + threads - 1) / threads;
   const int g = (int)(b < 1 ? 1 : (b > 148LL * 16 ? 148LL * 16 : b));
-  quant_weight_kernel<<<g, threads, 0, st>>>((const float4*)w, n_blocks, m0, m1, (uint32_t)remap_code, scale_in,
-                                             amax_scratch, (uint2*)codes, scales, scale_out);
+  if (scale_aware)
+    quant_weight_kernel<true><<<g, threads, 0, st>>>((const float4*)w, n_blocks, sub, m0, m1, (uint32_t)remap_code, scale_in,
+                                                     amax_scratch, (uint2*)codes, scales, scale_out);
+  else
+    quant_weight_kernel<false><<<g, threads, 0, st>>>((const float4*)w, n_blocks, sub, m0, m1, (uint32_t)remap_code, scale_in,
+                                                      amax_scratch, (uint2*)codes, scales, scale_out);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "quant_weight_kernel launch");
 }

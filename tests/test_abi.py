@@ -41,11 +41,13 @@ def test_host_side_validation(binding):
     b = binding
     good = b.make_desc(256, 512, 0.01)
     assert b.razer_packed_bytes(good) == 2 * 8 * 4608           # 2 row tiles x 8 k-chunks
+    assert b.razer_packed_bytes(b.make_desc(256, 512, 0.01, block=128)) == 2 * 8 * 4608   # one byte per 16 elements whatever the block
     assert b.razer_packed_bytes(b.make_desc(1, 16, 1.0)) == 4608  # padded to one tile-chunk
     for bad, code in [
         (b.make_desc(256, 520, 0.01), b.ERR_INVALID_ARG),                   # K % 16
         (b.make_desc(0, 512, 0.01), b.ERR_INVALID_ARG),
-        (b.make_desc(256, 512, 0.01, block=32), b.ERR_UNSUPPORTED),
+        (b.make_desc(256, 512, 0.01, block=48), b.ERR_UNSUPPORTED),
+        (b.make_desc(256, 544, 0.01, block=64), b.ERR_INVALID_ARG),                 # K % block
         (b.make_desc(256, 512, 0.01, sv_mag=(5.0, 8.5)), b.ERR_UNSUPPORTED),  # 8.5 is not exact in bf16 products
         (b.make_desc(256, 512, 0.01, remap_code=3), b.ERR_INVALID_ARG),
         (b.make_desc(256, 512, 0.0), b.ERR_INVALID_ARG),

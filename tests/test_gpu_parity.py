@@ -248,6 +248,61 @@ def test_quant_weight_bit_exact(b, N, K, seed, sv_mag, remap_code):
     assert np.linalg.norm(d2 - w.numpy()) / np.linalg.norm(w.numpy()) < 0.12
 
 
+@pytest.mark.parametrize("block", [32, 64, 128])
+def test_larger_blocks_quantize_pack_and_multiply(b, block):
+    """Block sizes 32 / 64 / 128 (Sec. 5's block-size study, Sec. 4.3's deployment size): the GPU weight quantizer
+    against the oracle's bit for bit (near-ties aside), the packed form's dequantization bit-exact, the decode
+    GEMV and the tensor-core GEMM within the matmul bars."""
+    N, K = 260, 2048
+    w = inputs.student_t_weights(N, K, 160 + block, outlier_frac=0.001)
+    codes, scales, ts = b.razer_quant_weight(w.cuda(), block=block)
+    torch.cuda.synchronize()
+    want_c, want_s, want_d, dbg = ro.quantize_weight(w.numpy(), block=block, return_debug=True)
+    assert np.float32(ts.item()) == want_d and tuple(scales.shape) == (N, K // block)
+    got_s, got_c = scales.cpu().numpy(), codes.cpu().numpy()
+    assert np.array_equal(got_s & 0x3F, want_s & 0x3F)
+    blk_ok = (got_s == want_s) & np.all((got_c == want_c).reshape(N, K // block, block // 2), axis=2)
+    assert np.all(blk_ok | dbg["near_tie"]) and blk_ok.mean() > 0.999
+    desc = b.make_desc(N, K, float(ts.item()), block=block)
+    packed = b.razer_pack_layout(desc, codes, scales)
+    d2 = b.razer_dequant(desc, packed, fp32=True).cpu().numpy()
+    want2 = ro.dequant_d2(got_c, got_s, np.float32(ts.item()), block=block)
+    assert np.array_equal(d2.view(np.uint32), want2.view(np.uint32))
+    for M, fn in ((1, b.razer_gemv), (40, b.razer_gemv), (130, b.razer_gemm)):
+        x = inputs.activations(M, K, 170 + M)
+        _check_matmul(b, fn, desc, packed, got_c, got_s, float(ts.item()), x, block=block)
+
+
+@pytest.mark.parametrize("N,K,seed,sv_mag,block", [(512, 1024, 21, (5.0, 8.0), 16), (200, 2048, 22, (7.0, 10.0), 32),
+                                                    (130, 528, 23, (2.5, 5.0), 16)])
+def test_quant_weight_scale_aware_bit_exact(b, N, K, seed, sv_mag, block):
+    """Scale-aware special-value selection (Eq. 6-7 with the scale of Eq. 2 chosen together with v) on the GPU
+    against the oracle's: same scale codes and metadata, same element codes, near-ties aside; the result decodes
+    through the unchanged kernels and is no worse than the plain selection's."""
+    w = inputs.student_t_weights(N, K, seed, outlier_frac=0.001)
+    codes, scales, ts = b.razer_quant_weight(w.cuda(), sv_mag=sv_mag, block=block, scale_aware=True)
+    torch.cuda.synchronize()
+    want_c, want_s, want_d, dbg = ro.quantize_scale_aware(w.numpy(), sv_mag=sv_mag, block=block, return_debug=True)
+    assert np.float32(ts.item()) == want_d
+    got_s, got_c = scales.cpu().numpy(), codes.cpu().numpy()
+    blk_ok = (got_s == want_s) & np.all((got_c == want_c).reshape(N, K // block, block // 2), axis=2)
+    assert np.all(blk_ok | dbg["near_tie"]) and blk_ok.mean() > 0.999
+    desc = b.make_desc(N, K, float(ts.item()), sv_mag=sv_mag, block=block)
+    packed = b.razer_pack_layout(desc, codes, scales)
+    d2 = b.razer_dequant(desc, packed, fp32=True).cpu().numpy()
+    want2 = ro.dequant_d2(got_c, got_s, np.float32(ts.item()), sv_mag=sv_mag, block=block)
+    assert np.array_equal(d2.view(np.uint32), want2.view(np.uint32))
+    c0, s0, t0 = b.razer_quant_weight(w.cuda(), sv_mag=sv_mag, block=block)
+    plain = ro.dequant_d2(c0.cpu().numpy(), s0.cpu().numpy(), np.float32(t0.item()), sv_mag=sv_mag, block=block)
+    e_aware, e_plain = np.linalg.norm(d2 - w.numpy()), np.linalg.norm(plain - w.numpy())
+    if max(sv_mag) > 6.0:
+        assert e_aware < e_plain
+    else:
+        assert np.array_equal(got_c, c0.cpu().numpy()) and np.array_equal(got_s, s0.cpu().numpy())
+    x = inputs.activations(3, K, seed + 100)
+    _check_matmul(b, b.razer_gemv, desc, packed, got_c, got_s, float(ts.item()), x, sv_mag=sv_mag, block=block)
+
+
 def test_quant_weight_given_scale_and_zero_input(b):
     w = inputs.student_t_weights(16, 256, 7)
     given = torch.tensor([0.01], dtype=torch.float32)

@@ -225,3 +225,122 @@ def test_w4a4_matmul_against_dequantized_product():
     # and the quantized product approximates the real one
     ref = x.double().numpy() @ w.astype(np.float64).T
     assert np.linalg.norm(y - ref) / np.linalg.norm(ref) < 0.2
+
+
+# --------------------------------------------------------------------------
+# block sizes 32 / 64 / 128 (the block-size study of Sec. 5; Sec. 4.3 deploys 128)
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("block", [32, 64, 128])
+def test_larger_blocks_scale_and_error_invariants(block):
+    """One scale and one special value per `block` elements: the scale follows Eq. 2 on the block's maximum, the
+    error with the special value never exceeds plain FP4 at the same scale (Q is a subset of Q + {v}), the decoded
+    block attains the error the encoder reported, and element-wise optimality holds given (scale, v): every code is
+    the nearest member of Q + {v}."""
+    w = _weights(64, 1024, 30 + block)
+    codes, scales, d32, dbg = ro.quantize(w, ro.SCALE_E3M3_META2, (5.0, 8.0), 0x8, block=block, return_debug=True)
+    nb = 1024 // block
+    assert scales.shape == (64, nb)
+    bmax = np.abs(w).reshape(64, nb, block).max(axis=2)
+    t = (bmax / np.float32(d32 * np.float32(6.0))).astype(np.float32)
+    want = ro.round_to_scale(t, ro.SCALE_E3M3_META2)
+    want = np.where((bmax > 0) & (want == 0), 1, want)
+    assert np.array_equal(scales & 0x3F, want)
+    e = dbg["errs64"]
+    assert np.all(e <= dbg["err_fp4"][None] + 1e-12)
+    chosen = np.take_along_axis(e, dbg["meta"][None].astype(np.int64), axis=0)[0]
+    assert np.all((chosen <= e.min(axis=0) * (1 + 1e-5) + 1e-12) | dbg["near_tie"])
+    q, s = ro.decode_block_values(codes, scales, block=block)
+    xs = dbg["xs"].reshape(64, 1024).astype(np.float64)
+    achieved = np.sum(((q - xs) ** 2).reshape(64, nb, block), axis=2)
+    assert np.allclose(achieved, chosen, rtol=1e-9, atol=1e-12)
+    # nearest member of Q + {v}, element by element (brute force over the 16 values)
+    sv = np.repeat(np.array(ro.sv_candidates((5.0, 8.0), ro.SCALE_E3M3_META2))[dbg["meta"]], block, axis=1)
+    fp4 = np.array(sorted({ro.fp4_value(c) for c in range(16)}))
+    d_best = np.minimum(np.min(np.abs(xs[:, :, None] - fp4[None, None, :]), axis=2), np.abs(xs - sv))
+    assert np.allclose(np.abs(q - xs), d_best, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("block", [32, 64, 128])
+def test_larger_blocks_decode_equals_block16_with_repeated_scale_bytes(block):
+    """A block of 16 k elements with one scale byte decodes exactly like k blocks of 16 that carry the same byte:
+    this is what lets the packed form keep one byte per 16 elements for every block size."""
+    w = _weights(32, 512, 40 + block)
+    codes, scales, d32 = ro.quantize(w, ro.SCALE_E3M3_META2, (5.0, 9.0), 0x0, block=block)
+    a = ro.dequant_d2(codes, scales, d32, sv_mag=(5.0, 9.0), remap_code=0x0, block=block)
+    b = ro.dequant_d2(codes, np.repeat(scales, block // 16, axis=1), d32, sv_mag=(5.0, 9.0), remap_code=0x0)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+    # and a larger block can only do worse than (or as well as) its 16-element sub-blocks quantized on their own
+    c16, s16, d16 = ro.quantize(w, ro.SCALE_E3M3_META2, (5.0, 9.0), 0x0, block=16, tensor_scale=d32)
+    e_big = np.sum((a.astype(np.float64) - w) ** 2)
+    e_16 = np.sum((ro.dequant_d2(c16, s16, d16, sv_mag=(5.0, 9.0), remap_code=0x0).astype(np.float64) - w) ** 2)
+    assert e_16 <= e_big * 1.02
+
+
+# --------------------------------------------------------------------------
+# scale-aware special-value selection (Eq. 6-7 with the scale of Eq. 2 chosen together with v)
+# --------------------------------------------------------------------------
+
+def _err_in_tensor_units(w, codes, scales, d32, **kw):
+    d2 = ro.dequant_d2(codes, scales, d32, **kw).astype(np.float64)
+    return ((d2 - w.astype(np.float64)) ** 2).reshape(w.shape[0], -1, 16).sum(axis=2)
+
+
+def test_scale_aware_reaches_a_special_value_beyond_six_exactly():
+    """A block that is exactly s * [8, 1, -2, 3, 0.5, ...]: with Eq. 2's Qmax = 6 the 8 cannot be hit (the scale
+    makes it 6 and the rest moves off the grid); with the scale chosen for v = 8 the block is reproduced exactly."""
+    vals = np.array([8, 1, -2, 3, 0.5, -1.5, 4, 6, 0, -0.5, 2, -3, 1, 1.5, -4, 0.5], dtype=np.float32)
+    s = np.float32(ro.e4m3_value(20))                              # a scale in the middle of the E3M3 grid
+    w = np.stack([vals * s, -vals * s]).astype(np.float32)
+    d32 = np.float32(1.0)
+    c, sc, _ = ro.quantize_scale_aware(w, tensor_scale=d32)
+    assert np.array_equal(ro.dequant_d2(c, sc, d32), w)            # exact, for +8 and for -8
+    assert list(sc >> 6) == [[1], [3]] and list(sc & 0x3F) == [[20], [20]]
+    c0, s0, _ = ro.quantize_weight(w, tensor_scale=d32)
+    assert _err_in_tensor_units(w, c0, s0, d32).min() > 0          # the plain selection cannot
+
+
+def test_scale_aware_never_worse_and_identical_without_large_special_values():
+    w = _weights(96, 512, 50)
+    c1, s1, d1, dbg = ro.quantize_scale_aware(w, return_debug=True)
+    c0, s0, d0 = ro.quantize_weight(w)
+    assert d0 == d1
+    e1, e0 = _err_in_tensor_units(w, c1, s1, d1), _err_in_tensor_units(w, c0, s0, d0)
+    assert np.all((e1 <= e0 * (1 + 1e-5) + 1e-18) | dbg["near_tie"])      # a superset of candidates
+    assert e1.sum() < e0.sum()                                           # and +-8 now does get used
+    used8 = ((s1 >> 6) & 1) == 1
+    assert used8.mean() > ((s0 >> 6) & 1).mean()
+    # the reported minimum is what the decoded block has
+    got = np.take_along_axis(dbg["errs64"], dbg["pick"][None], axis=0)[0]
+    assert np.allclose(e1, got, rtol=1e-4, atol=1e-16)     # xs is rounded to FP32 on the way
+    # no special value beyond 6: the candidate list is the plain one, the result identical
+    a = ro.quantize_scale_aware(w, sv_mag=(2.5, 5.0))
+    b = ro.quantize_weight(w, sv_mag=(2.5, 5.0))
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))
+
+
+def test_scale_aware_brute_force_over_its_candidates_on_tiny_blocks():
+    """Blocks of two elements: for every (special value, scale) candidate the method allows, enumerate all 256 code
+    vectors; the encoder's choice attains the minimum of the reconstruction error over all of them."""
+    rng = np.random.default_rng(11)
+    w = (rng.standard_t(5, size=(30, 8)) * 0.02).astype(np.float32)
+    c, s, d32 = ro.quantize_scale_aware(w, block=2)
+    q, sv = ro.decode_block_values(c, s, block=2)
+    got = (((q * np.repeat(sv, 2, axis=1) * float(d32)) - w) ** 2).reshape(30, 4, 2).sum(axis=2)
+    cands = ro.sv_candidates((5.0, 8.0), ro.SCALE_E3M3_META2)
+    grid = ro.scale_grid(ro.SCALE_E3M3_META2)
+    wb = w.reshape(30, 4, 2).astype(np.float64)
+    for r in range(30):
+        for b in range(4):
+            bmax = np.abs(wb[r, b]).max()
+            top_neg = wb[r, b][np.argmax(np.abs(wb[r, b]))] < 0
+            best = np.inf
+            for v in cands:
+                for qmax in ([6.0, abs(v)] if abs(v) > 6 and (v < 0) == top_neg else [6.0]):
+                    t = np.float32(np.float32(bmax) / np.float32(d32 * np.float32(qmax)))
+                    sc = max(int(ro.round_to_scale(np.array([t]), ro.SCALE_E3M3_META2)[0]), 1)
+                    step = float(np.float32(d32 * np.float32(grid[sc])))
+                    vals = np.array([ro.fp4_value(k) if k != 8 else v for k in range(16)]) * step
+                    e = (vals[:, None] - wb[r, b][None, :]) ** 2       # [16 values, 2 elements]
+                    best = min(best, e[:, 0].min() + e[:, 1].min())
+            assert got[r, b] <= best * (1 + 1e-4) + 1e-18      # midpoint decisions are taken on FP32-rounded xs
