@@ -189,6 +189,29 @@ def run_reference(args):
     }))
 
 
+def run_shape(args):
+    """One matmul shape alone: `warmup` launches, then `steps` launches timed with CUDA events, two packed copies
+    of the weights in turn.  M <= 64 goes through razer_gemv, larger M through razer_gemm."""
+    import torch
+    from paper_2501_04052_b200 import build
+    build.build()
+    from paper_2501_04052_b200 import binding as b
+    from paper_2501_04052_b200 import inputs
+    M, N, K = (int(v) for v in args.shape.lower().split("x"))
+    desc, sets, _ = make_sets(b, torch, inputs, N, K, 2, 7)
+    x = inputs.activations(M, K, 3).cuda()
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    fn, op = (b.razer_gemv, b.OP_GEMV) if M <= 64 else (b.razer_gemm, b.OP_GEMM)
+    ws = b.alloc_workspace(desc, M, op, "cuda")
+    for i in range(args.warmup):
+        fn(desc, sets[i % 2], x, y, ws)
+    ms = time_cuda(lambda i: fn(desc, sets[i % 2], x, y, ws), args.steps, torch)
+    b.razer_workspace_status(ws)
+    print(json.dumps({"shape": [M, N, K], "op": "razer_gemv" if M <= 64 else "razer_gemm", "us_per_launch_stream": ms * 1e3,
+                      "launches": args.warmup + args.steps, "algorithmic_bytes": algo_bytes(M, N, K),
+                      "flops": 2.0 * M * N * K}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -199,9 +222,13 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--windows", type=int, default=7, help="timed windows (the median is reported)")
     ap.add_argument("--window-ms", type=float, default=200.0, help="length of a timed window (0: one graph replay)")
+    ap.add_argument("--shape", default="", help="MxNxK: time that one matmul alone (a small, single-kernel run for "
+                                                "profiler captures); prints its own short JSON line, not the bench line")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.shape:
+        return run_shape(args)
 
     import torch
     from paper_2501_04052_b200 import build

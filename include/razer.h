@@ -162,7 +162,8 @@ int razer_gemv_static(const razer_desc* d, const void* packed_dev, const void* x
 
 /* Online activation quantization (Sec. 4.2: each block is quantized once per allowed
  * special value, +sv_mag and -sv_mag, and the lower squared error wins; Eq. 1-3, 6-7 with
- * the 7-bit E4M3 block scale).  x_dev: bf16 [M][K], K multiple of 16.
+ * the 7-bit E4M3 block scale).  sv_mag = 0 quantizes to plain NVFP4 (Eq. 1-3 alone: no special
+ * value, metadata bit clear).  x_dev: bf16 [M][K], K multiple of 16.
  * tensor_scale_in_dev: device float to use as the Eq. 1 scale, or NULL to compute it from
  * the tensor maximum.  In that case amax_scratch_dev is required: two device uint32 (8-byte
  * aligned) that are ZERO before the first call; every call leaves them zero again, so one
@@ -204,10 +205,21 @@ int razer_quant_weight(const float* w_dev, int N, int K, int block, int scale_aw
 int razer_decode_act(const uint8_t* act_codes_dev, const uint8_t* act_scales_dev, int M, int K,
                      float sv_mag, void* out_bf16_dev, void* stream);
 
-/* Weight-activation GEMM (App. D.3 setting, both operands RaZeR):
+/* Weight-activation GEMM (App. D.3 setting):
  * y = bf16( w_scale * a_scale * sum_k decoded_act[m][k] * decoded_w[n][k] ).
- * The workspace (RAZER_OP_GEMM_W4A4) holds the decoded activations.
- * use_native_fp4 must be 0 in this build (block-scaled FP4 MMA path not present). */
+ * act_codes_dev [M][K/2], act_scales_dev [M][K/16], act_tensor_scale_dev: one device float, as
+ * razer_quant_act writes them.  The workspace (RAZER_OP_GEMM_W4A4, zeroed once by
+ * razer_workspace_init, 256-byte aligned) serves either path below.
+ * use_native_fp4 = 0: both operands RaZeR; the activations are decoded to bf16 (exact) into the
+ * workspace and multiplied by the bf16 tensor-core kernel of razer_gemm.
+ * use_native_fp4 != 0: the two-pass realization of App. D.3 on the block-scaled FP4 tensor-core
+ * instruction (block 16, E4M3 scale factors): the weights are split on the fly into B_main
+ * (special value -> signed FP4 base value) and B_comp (signed FP4 remainder, zero elsewhere),
+ * both passes accumulate in FP32 into the same accumulator.  RaZeR applies to the weights only:
+ * the activations are read as plain NVFP4 (act_sv_mag is ignored, bit 7 of a scale byte is
+ * ignored and code 0x8 is a zero), which is what razer_quant_act writes with sv_mag = 0.  Both
+ * special-value magnitudes of the descriptor must be sums of two FP4 values (every allowed
+ * magnitude is).  Two kernel launches (activation re-layout, matmul). */
 int razer_gemm_w4a4(const razer_desc* d, const void* packed_w_dev, const uint8_t* act_codes_dev,
                     const uint8_t* act_scales_dev, const float* act_tensor_scale_dev, float act_sv_mag,
                     int M, void* y_dev, void* workspace_dev, size_t workspace_bytes,

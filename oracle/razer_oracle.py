@@ -227,7 +227,7 @@ def quantize(x: np.ndarray, scale_fmt: int = SCALE_E3M3_META2, sv_mag=(5.0, 8.0)
     f32 = np.float32
     grid = scale_grid(scale_fmt) * (2.0 ** scale_bias_shift)
     smax = f32(grid[-1])
-    cands = sv_candidates(sv_mag, scale_fmt)
+    cands = sv_candidates(sv_mag, scale_fmt) if sv_mag is not None else []   # None: plain NVFP4, Eq. 1-3 alone
     mbits = meta_bits(scale_fmt)
     shift = 8 - mbits
 
@@ -270,8 +270,12 @@ def quantize(x: np.ndarray, scale_fmt: int = SCALE_E3M3_META2, sv_mag=(5.0, 8.0)
         d64 = q.astype(np.float64) - xs.astype(np.float64)
         errs64[ci] = np.sum(d64 * d64, axis=2)
         use_sv[ci] = take
-    meta = np.argmin(errs32, axis=0).astype(np.uint8)          # first minimum = smallest meta
-    take = np.take_along_axis(use_sv, meta[None, :, :, None].astype(np.int64), axis=0)[0]
+    if cands:
+        meta = np.argmin(errs32, axis=0).astype(np.uint8)      # first minimum = smallest meta
+        take = np.take_along_axis(use_sv, meta[None, :, :, None].astype(np.int64), axis=0)[0]
+    else:                                                      # no special value: every element keeps r(xs)
+        meta = np.zeros((R, nb), dtype=np.uint8)
+        take = np.zeros((R, nb, block), dtype=bool)
 
     other_zero = remap_code ^ 0x8
     std_code = (ridx | (np.signbit(xs).astype(np.uint8) << 3)).astype(np.uint8)
@@ -285,7 +289,8 @@ def quantize(x: np.ndarray, scale_fmt: int = SCALE_E3M3_META2, sv_mag=(5.0, 8.0)
     if return_debug:
         d0 = rval.astype(np.float64) - xs.astype(np.float64)
         dbg = dict(xs=xs, errs32=errs32, errs64=errs64, err_fp4=np.sum(d0 * d0, axis=2),
-                   meta=meta, scode=scode, near_tie=_near_ties(errs64))
+                   meta=meta, scode=scode,
+                   near_tie=_near_ties(errs64) if len(cands) > 1 else np.zeros((R, nb), dtype=bool))
         return packed, sbyte, d32, dbg
     return packed, sbyte, d32
 
@@ -397,9 +402,11 @@ def quantize_weight(w, sv_mag=(5.0, 8.0), remap_code=0x8, **kw):
 
 def quantize_act(x_bf16_bits, sv_mag=(5.0,), remap_code=0x8, tensor_scale=None, **kw):
     """Online activation quantization (Sec. 4.2, "double quantization"): bf16 input
-    widened to FP32, E4M3 block scale, two special values +-sv_mag[0]."""
+    widened to FP32, E4M3 block scale, two special values +-sv_mag[0].  sv_mag = None
+    gives plain NVFP4 (Sec. 3, Eq. 1-3), the activation format of the two-pass tensor-core
+    realization (App. D.3)."""
     x = bf16_bits_to_f32(x_bf16_bits)
-    return quantize(x, SCALE_E4M3_META1, (sv_mag[0], sv_mag[0]), remap_code,
+    return quantize(x, SCALE_E4M3_META1, None if sv_mag is None else (sv_mag[0], sv_mag[0]), remap_code,
                     tensor_scale=tensor_scale, **kw)
 
 

@@ -14,7 +14,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librazer.so")
-SOURCES = ["razer_api.cu", "razer_pack.cu", "razer_quant.cu", "razer_gemv_simt.cu", "razer_gemm_umma.cu", "razer_gemv_stream.cu",
+SOURCES = ["razer_api.cu", "razer_pack.cu", "razer_quant.cu", "razer_gemv_simt.cu", "razer_gemm_umma.cu", "razer_gemm_fp4.cu", "razer_gemv_stream.cu",
            "razer_static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]

@@ -73,6 +73,9 @@ int launch_quant_act(const void*, int, int, float, const float*, uint32_t*, uint
 int launch_gemv_simt(const razer_desc*, const void*, const void*, int, const float*, void*, void*, size_t,
                      cudaStream_t);
 size_t simt_workspace_bytes(const razer_desc*, int M);
+int launch_gemm_fp4(const razer_desc*, const void*, const uint8_t*, const uint8_t*, const float*, int, void*, void*, size_t,
+                    cudaStream_t);
+size_t gemm_fp4_workspace_bytes(const razer_desc*, int M);
 int launch_gemm_umma(const razer_desc*, const void* packed, const void* x, int M, int ldx_K, float extra_scale,
                      const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
 size_t umma_workspace_bytes(const razer_desc*, int M);
@@ -162,7 +165,9 @@ int razer_workspace_bytes(const razer_desc* d, int M, int op, size_t* bytes_out)
       break;
     case RAZER_OP_GEMM_W4A4: {
       const size_t g = matmul_workspace_need(d, M);
-      b = align_up((size_t)M * d->K * 2, 256) + g;
+      b = align_up((size_t)M * d->K * 2, 256) + g;                     // decoded activations + the bf16 matmul's own
+      const size_t f = gemm_fp4_workspace_bytes(d, M);                 // or the block-scaled FP4 path's
+      b = b > f ? b : f;
       break;
     }
     default:
@@ -255,7 +260,8 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag, const float* 
                     uint32_t* amax_scratch_dev, uint8_t* act_codes_dev, uint8_t* act_scales_dev,
                     float* tensor_scale_out_dev, void* stream) {
   if (M < 1 || K < 16 || K % 16) return set_error(RAZER_ERR_INVALID_ARG, "M=%d K=%d invalid (K %% 16 == 0)", M, K);
-  if (!sv_allowed(sv_mag)) return set_error(RAZER_ERR_UNSUPPORTED, "special value magnitude %g is not allowed", sv_mag);
+  if (sv_mag != 0.0f && !sv_allowed(sv_mag))                           // 0: no special value (plain NVFP4)
+    return set_error(RAZER_ERR_UNSUPPORTED, "special value magnitude %g is not allowed", sv_mag);
   RAZER_TRY(check_ptr(x_dev, 16, "x_dev"));
   RAZER_TRY(check_ptr(act_codes_dev, 8, "act_codes_dev"));
   RAZER_TRY(check_ptr(act_scales_dev, 1, "act_scales_dev"));
@@ -302,9 +308,16 @@ int razer_gemm_w4a4(const razer_desc* d, const void* packed_w_dev, const uint8_t
                     void* y_dev, void* workspace_dev, size_t workspace_bytes, int use_native_fp4, void* stream) {
   RAZER_TRY(check_desc(d));
   if (M < 1) return set_error(RAZER_ERR_INVALID_ARG, "M=%d must be positive", M);
-  if (use_native_fp4) return set_error(RAZER_ERR_UNSUPPORTED, "the block-scaled FP4 MMA path is not built");
   RAZER_TRY(check_ptr(act_tensor_scale_dev, 4, "act_tensor_scale_dev"));
   RAZER_TRY(check_ptr(workspace_dev, 256, "workspace_dev"));
+  if (use_native_fp4) {
+    RAZER_TRY(check_ptr(packed_w_dev, 16, "packed_w_dev"));
+    RAZER_TRY(check_ptr(act_codes_dev, 8, "act_codes_dev"));
+    RAZER_TRY(check_ptr(act_scales_dev, 1, "act_scales_dev"));
+    RAZER_TRY(check_ptr(y_dev, 2, "y_dev"));
+    return launch_gemm_fp4(d, packed_w_dev, act_codes_dev, act_scales_dev, act_tensor_scale_dev, M, y_dev, workspace_dev,
+                           workspace_bytes, (cudaStream_t)stream);
+  }
   const size_t act_bytes = align_up((size_t)M * d->K * 2, 256);
   if (workspace_bytes < act_bytes) return set_error(RAZER_ERR_WORKSPACE, "workspace too small for the decoded activations");
   cudaStream_t st = (cudaStream_t)stream;

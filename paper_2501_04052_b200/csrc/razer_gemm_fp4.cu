@@ -1,0 +1,660 @@
+// Two-pass block-scaled FP4 matmul of RaZeR weights against plain-NVFP4 activations (App. D.3) on the
+// 5th-generation tensor core (tcgen05.mma kind::mxf4nvf4, block 16, UE4M3 scale factors).
+//
+//   y[m, n] = bf16( ts_w * ts_a * sum_k A[m, k] * (B_main[n, k] + B_comp[n, k]) )
+//
+// B_main keeps every ordinary code and puts a signed FP4 base value where the block's special value sits,
+// B_comp holds the signed FP4 remainder there and zero elsewhere (base + remainder = special value).  Both
+// share the block's scale byte: the 6-bit E3M3 code is an E4M3 code with a clear top bit, so the masked byte
+// is the hardware's UE4M3 scale factor as it stands.  The two passes are two MMAs per 64-column chunk into
+// the same TMEM accumulator; neither matrix exists in global memory.
+//
+// Mapping: the weight tile is the MMA's A operand (128 rows), the token tile its B operand (128 tokens),
+// both K-major FP4 in shared memory with the 128-byte swizzle (one row = 256 codes = one stage of four
+// chunks).  Warp 0 = TMA producer (packed weights, activation codes, activation scale factors), warp 1 =
+// TMEM owner and MMA issuer, warps 2..9 = remap (thread = weight row; two groups of four warps take the
+// stages in turn) and epilogue.  A remap thread reads its row's packed blocks, finds the special-value
+// nibbles (the only nibbles that are 0x0 in the packed form), builds the two code words with two integer
+// multiply-adds, applies the block's stored-negated flag to the sign bits, and writes both rows plus the row's
+// four scale bytes (scale-factor layout: 32 x 16-byte rows, row r % 32, word r / 32).  The MMA warp copies
+// the scale factors of both operands to TMEM (tcgen05.cp) and issues main and comp MMAs.
+//
+// The activation operand is prepared by a small kernel before the matmul: codes padded to whole stages with
+// the nibbles of every 32-bit word in the packed form's order (the contraction does not care about the order
+// of k inside a block as long as both operands agree), scale bytes masked to 7 bits and laid out as the
+// scale-factor tiles the MMA reads.
+//
+// Work partition, partial tiles and bounded waits are those of the bf16 tcgen05 kernel: a persistent grid,
+// contiguous stripes of (tile, stage) items, partial tiles through FP32 slots and a per-tile counter.
+#include <cuda.h>
+#include <cstdlib>
+
+#include "razer_common.cuh"
+#include "razer_ptx.cuh"
+#include "razer_tcgen05.cuh"
+
+namespace razer {
+namespace fp4_path {
+
+constexpr int NT = 128;                               // tokens per tile (MMA N)
+constexpr int CH = 4;                                 // chunks per stage: 256 codes = one 128-byte swizzled row
+constexpr int STAGES = 4;                             // shared-memory ring fed by TMA
+constexpr int ASTAGES = 2;                            // remapped-operand ring, one slot per remap group
+constexpr int NRW = 8;                                // remap warps
+constexpr int THREADS = 64 + 32 * NRW;
+constexpr int W_BYTES = CH * CHUNK_BYTES;             // 18432 packed weight bytes of a stage
+constexpr int X_BYTES = NT * 128;                     // activation codes of a stage
+constexpr int SF_TILE_BYTES = 512;                    // scale factors of 128 rows x one chunk
+constexpr int SF_BYTES = CH * SF_TILE_BYTES;
+constexpr int STAGE_BYTES = W_BYTES + X_BYTES + SF_BYTES;
+constexpr int A_TILE_BYTES = TILE_ROWS * 128;         // 128 rows x 256 codes
+constexpr int ASTAGE_BYTES = 2 * A_TILE_BYTES + SF_BYTES;
+constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 4;
+constexpr int ACC_COLS = NT;
+constexpr int SF_COLS = 2 * CH * 4;                   // per operand ring slot: A and B scale factors of four chunks
+constexpr int TMEM_COLS = 256;
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + (size_t)ASTAGES * ASTAGE_BYTES + NUM_BARS * 8 + 64;
+static_assert(STAGE_BYTES % 1024 == 0 && W_BYTES % 1024 == 0 && ASTAGE_BYTES % 1024 == 0, "swizzled tiles sit on 1024 bytes");
+static_assert(ACC_COLS + ASTAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+
+struct Args {
+  __nv_bfloat16* y;
+  const uint8_t* sfb;        // activation scale factors: [token tile][stage][chunk] tiles of 512 bytes
+  float* slots;              // [grid][2][NT][128] FP32 partial tiles
+  uint32_t* counters;        // one per output tile, zero between calls
+  uint32_t* status;          // device status word
+  const float* extra_scale;  // device scalar multiplied into the tensor scale (the activations' tensor scale)
+  Geometry g;
+  float tensor_scale;
+  uint32_t base0, rem0, base1, rem1;   // FP4 codes of the base value and the remainder for select 0 / 1
+  int M, token_tiles, steps_per_tile;
+  long long total_items;
+};
+
+// D[tmem] (+)= A[smem] * B[smem], FP4 operands with one UE4M3 scale factor per 16 elements read from TMEM.
+__device__ __forceinline__ void mma_fp4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                        uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+      "setp.ne.b32 p, %7, 0;\n\t"
+      "mov.b64 ad, {%1, %3};\n\t"
+      "mov.b64 bd, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], ad, bd, %4, [%5], [%6], p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+// 32 rows x 16 bytes of shared memory -> 4 TMEM columns, the same in all four 32-lane quarters.
+__device__ __forceinline__ void copy_sf_to_tmem(uint32_t tmem, uint32_t saddr) {
+  // no swizzle; eight 16-byte rows are contiguous, groups of eight rows 128 bytes apart
+  const uint32_t lo = (saddr & 0x3FFFFu) >> 4;
+  const uint32_t hi = (128u >> 4) | (1u << 14);
+  asm volatile(
+      "{\n\t.reg .b64 sd;\n\t"
+      "mov.b64 sd, {%1, %2};\n\t"
+      "tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], sd;\n\t}" ::"r"(tmem),
+      "r"(lo), "r"(hi)
+      : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+// writes made through the generic proxy become visible to the tensor core's (asynchronous proxy) reads
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Instruction descriptor: E2M1 x E2M1 -> FP32, UE4M3 scale factors, both operands K-major, M = 128, N = NT.
+constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// Upper half of an operand's shared-memory descriptor: 1024-byte group stride, descriptor version, 128-byte swizzle.
+constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+
+__global__ void __launch_bounds__(THREADS, 1)
+razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Args a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem_a = smem + (size_t)STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_a + (size_t)ASTAGES * ASTAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  uint32_t* bcast = tmem_slot + 2;
+
+  const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> remap, MMA
+  const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]  MMA commit -> TMA
+  const uint32_t bar_afull = bar_empty + 8 * STAGES;    // [ASTAGES] remap -> MMA
+  const uint32_t bar_aempty = bar_afull + 8 * ASTAGES;  // [ASTAGES] MMA commit -> remap
+  const uint32_t bar_accfull = bar_aempty + 8 * ASTAGES;
+  const uint32_t bar_accempty = bar_accfull + 8;
+  const uint32_t bar_epi = bar_accempty + 8;            // rendezvous of the epilogue threads
+  const uint32_t bar_drain = bar_epi + 8;               // the MMA warp's own MMAs have all completed
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grid = gridDim.x, cta = blockIdx.x;
+  const int it_begin = (int)((a.total_items * cta) / grid);
+  const int it_end = (int)((a.total_items * (cta + 1)) / grid);
+  const int n_items = it_end - it_begin;
+  const int spt = a.steps_per_tile;
+  ItemCursor cur;
+  cur.tile = it_begin / spt;
+  cur.step = it_begin - cur.tile * spt;
+  cur.stage = cur.phase = cur.astage = cur.aphase = 0;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < ASTAGES; ++i) {
+      mbar_init(bar_afull + 8 * i, 128);
+      mbar_init(bar_aempty + 8 * i, 1);
+    }
+    mbar_init(bar_accfull, 1);
+    mbar_init(bar_accempty, 32 * NRW);
+    mbar_init(bar_epi, 32 * NRW);
+    mbar_init(bar_drain, 1);
+    *abort_flag = 0;
+    tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // Producer state (thread 0 only).  The first ring of weight loads goes out before the rest of the prologue;
+  // the activation side (written by the preparation kernel) follows once that kernel has finished.
+  int issued = 0;
+  int p_rt = cur.tile / a.token_tiles, p_tt = cur.tile - p_rt * a.token_tiles;
+  auto produce_x = [&](int stage, int step, int tt) {
+    const uint32_t st = smem_u32(smem) + (uint32_t)stage * STAGE_BYTES;
+    const uint32_t bar = bar_full + 8 * stage;
+    tma_load_2d(st + W_BYTES, &tmap_x, step * 128, tt * NT, bar);
+    bulk_copy_g2s(st + W_BYTES + X_BYTES, a.sfb + ((size_t)tt * spt + step) * SF_BYTES, SF_BYTES, bar);
+  };
+  auto produce = [&](bool with_x) {
+    const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * STAGE_BYTES;
+    const uint32_t bar = bar_full + 8 * cur.stage;
+    // the weight box always spans CH chunks (zero-filled past the end of K)
+    mbar_expect_tx(bar, (uint32_t)(W_BYTES + X_BYTES + SF_BYTES));
+    tma_load_3d(st, &tmap_w, 0, cur.step * CH, p_rt * TILE_STRIPS, bar);
+    if (with_x) produce_x(cur.stage, cur.step, p_tt);
+    if (cur.step == spt - 1 && ++p_tt == a.token_tiles) { p_tt = 0; ++p_rt; }
+    cur.template next<STAGES, ASTAGES>(spt);
+  };
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_w) : "memory");
+    grid_dep_launch();
+    const ItemCursor first = cur;
+    const int first_tt = p_tt;
+    for (; issued < n_items && issued < STAGES; ++issued) produce(false);
+    grid_dep_wait();
+    ItemCursor c2 = first;
+    int tt2 = first_tt;
+    for (int i = 0; i < issued; ++i) {
+      produce_x(c2.stage, c2.step, tt2);
+      if (c2.step == spt - 1 && ++tt2 == a.token_tiles) tt2 = 0;
+      c2.template next<STAGES, ASTAGES>(spt);
+    }
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_sf0 = tmem_base + ACC_COLS;
+
+  auto fail = [&](uint32_t code) {
+    *abort_flag = 1;
+    grid_dep_wait();                                      // the status word lives in the (possibly shared) workspace
+    atomicCAS(a.status, 0u, code);
+  };
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      for (; issued < n_items; ++issued) {
+        if (!mbar_wait(bar_empty + 8 * cur.stage, (uint32_t)cur.phase ^ 1u, abort_flag)) { fail(21); break; }
+        produce(true);
+      }
+      // copies still in flight must land before this CTA's shared memory is released
+      const int pending = issued < STAGES ? issued : STAGES;
+      for (int f = issued - pending; f < issued; ++f)
+        mbar_wait(bar_full + 8 * (f % STAGES), (uint32_t)((f / STAGES) & 1), tmem_slot + 3);
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer (whole warp walks the items, one elected lane issues) =====================
+    uint32_t seg = 0;
+    auto wait_warp = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
+      const bool got = mbar_wait(bar, parity, abort_flag);
+      if (!got) fail(code);
+      return __all_sync(0xFFFFFFFFu, got);
+    };
+    for (int i = 0; i < n_items; ++i) {
+      const bool seg_first = (i == 0) || cur.step == 0;
+      const bool seg_last = (i + 1 == n_items) || cur.step == spt - 1;
+      const int nch = min(CH, a.g.k_chunks - cur.step * CH);
+      // the group that filled this operand slot waited for the shared-memory stage before it read it, so its
+      // arrival also covers the stage's activation codes and scale factors
+      if (!wait_warp(bar_afull + 8 * cur.astage, (uint32_t)cur.aphase, 23)) break;
+      if (seg_first && !wait_warp(bar_accempty, (seg & 1u) ^ 1u, 24)) break;
+      tc_fence_after();
+      const uint32_t xs = smem_u32(smem) + (uint32_t)cur.stage * STAGE_BYTES + W_BYTES;
+      const uint32_t sfb_s = xs + X_BYTES;
+      const uint32_t am = smem_u32(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES;
+      const uint32_t ac = am + A_TILE_BYTES;
+      const uint32_t sfa_s = am + 2 * A_TILE_BYTES;
+      const uint32_t sf_t = tmem_sf0 + cur.astage * SF_COLS;
+      if (elect_one()) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+          if (c < nch) {
+            const uint32_t sfa_t = sf_t + c * 4, sfb_t = sf_t + CH * 4 + c * 4;
+            copy_sf_to_tmem(sfa_t, sfa_s + c * SF_TILE_BYTES);
+            copy_sf_to_tmem(sfb_t, sfb_s + c * SF_TILE_BYTES);
+            // 64 codes further along k: +32 bytes inside the 128-byte rows
+            const uint32_t b_lo = ((xs + c * 32) >> 4) | (1u << 16);
+            mma_fp4(tmem_base, ((am + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t,
+                    (seg_first && c == 0) ? 0u : 1u);
+            mma_fp4(tmem_base, ((ac + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t, 1u);
+          }
+        }
+        tc_commit(bar_empty + 8 * cur.stage);
+        tc_commit(bar_aempty + 8 * cur.astage);
+        if (seg_last) tc_commit(bar_accfull);
+      }
+      __syncwarp();
+      if (seg_last) ++seg;
+      cur.template next<STAGES, ASTAGES>(spt);
+    }
+    // the MMAs issued so far read shared memory and TMEM until they complete: wait for them (bounded, not
+    // watching the abort flag) before the CTA may release either
+    __syncwarp();
+    if (elect_one()) tc_commit(bar_drain);
+    __syncwarp();
+    mbar_wait(bar_drain, 0u, tmem_slot + 3);
+  } else {
+    // ===================== remap (thread = weight row) + epilogue =====================
+    const int row = 32 * (warp & 3) + lane;              // weight row of the tile = TMEM lane of its outputs
+    const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
+    const int group = (warp - 2) >> 2;
+    constexpr int GROUPS = NRW / 4;
+    static_assert(GROUPS == ASTAGES && STAGES >= ASTAGES, "an operand slot per group; see the wait order below");
+    const int col_lo = 16 * ((group * (NT / 16)) / GROUPS);
+    const int col_hi = 16 * (((group + 1) * (NT / 16)) / GROUPS);
+    const bool leader = (threadIdx.x == 64);
+    float ts = a.tensor_scale;
+    bool dep_waited = false;
+    uint32_t seg = 0, epi_phase = 0;
+    auto wait_all = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
+      const bool got = mbar_wait(bar, parity, abort_flag);
+      if (!got) fail(code);
+      return __all_sync(0xFFFFFFFFu, got);
+    };
+    auto epi_sync = [&]() -> bool {
+      mbar_arrive(bar_epi);
+      const bool got = wait_all(bar_epi, epi_phase & 1u, 28);
+      ++epi_phase;
+      return got;
+    };
+    const int r16 = row % STRIP_ROWS;
+    const uint32_t strip_off = (uint32_t)(row / STRIP_ROWS) * (CH * PIECE_BYTES);
+    const uint32_t scale_off = (uint32_t)PIECE_CODE_BYTES + (uint32_t)(r16 & 7) * 8;
+    const uint32_t scale_sel = (r16 >> 3) ? 0x7531u : 0x6420u;
+    uint32_t code_off[CHUNK_BLOCKS];
+#pragma unroll
+    for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) code_off[blk] = (uint32_t)piece_code_offset(blk, r16);
+    const uint32_t row_off = (uint32_t)row * 128;        // this row inside an operand tile
+    const uint32_t sw7 = (uint32_t)row & 7u;              // 128-byte swizzle: 16-byte unit u of row r sits at u ^ (r % 8)
+    const uint32_t sf_word = (uint32_t)((row & 31) * 4 + (row >> 5)) * 4;
+    int turn = 0;                                        // item i is remapped by group i % GROUPS
+    for (int i = 0; i < n_items; ++i, cur.template next<STAGES, ASTAGES>(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
+      const int tile = cur.tile, step = cur.step;
+      const bool seg_last = (i + 1 == n_items) || step == spt - 1;
+      const int nch = min(CH, a.g.k_chunks - step * CH);
+      if (turn == group) {
+        // The operand slot is this group's own, and its release by the MMA warp (which takes the items in
+        // order) means that every item up to i - ASTAGES was issued, hence remapped, hence landed: the stage's
+        // previous fill (item i - STAGES, STAGES >= ASTAGES) among them, so the parity wait on it is sound.
+        if (!wait_all(bar_aempty + 8 * cur.astage, (uint32_t)cur.aphase ^ 1u, 26)) break;
+        if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 25)) break;
+        const uint32_t st = smem_addr(smem) + (uint32_t)cur.stage * STAGE_BYTES + strip_off;
+        const uint32_t am = smem_addr(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES + row_off;
+        const uint32_t ac = am + A_TILE_BYTES;
+        const uint32_t sfa = smem_addr(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES + 2 * A_TILE_BYTES + sf_word;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+          if (c < nch) {
+            const uint32_t ck = st + c * PIECE_BYTES;
+            const uint2 sq = lds64(ck + scale_off);
+            const uint32_t sw = __byte_perm(sq.x, sq.y, scale_sel);   // this row's four scale bytes, in block order
+            uint2 cw[CHUNK_BLOCKS];
+#pragma unroll
+            for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) cw[blk] = lds64(ck + code_off[blk]);
+            uint32_t mw[8], pw[8];
+#pragma unroll
+            for (int blk = 0; blk < CHUNK_BLOCKS; ++blk) {
+              const uint32_t sb = (sw >> (8 * blk)) & 0xFFu;
+              const uint32_t neg8 = (sb & PACKED_NEGATE) ? 0x88888888u : 0u;   // stored negated: flip every sign bit
+              const uint32_t base = (sb & PACKED_SELECT) ? a.base1 : a.base0;
+              const uint32_t rem = (sb & PACKED_SELECT) ? a.rem1 : a.rem0;
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const uint32_t w = h ? cw[blk].y : cw[blk].x;
+                const uint32_t any = w | (w >> 1) | (w >> 2) | (w >> 3);
+                const uint32_t z = ~any & 0x11111111u;                         // 1 in every nibble that is 0x0
+                mw[2 * blk + h] = (w + z * base) ^ neg8;
+                pw[2 * blk + h] = (z * rem) ^ neg8;
+              }
+            }
+            const uint32_t u0 = ((uint32_t)(2 * c) ^ sw7) << 4, u1 = ((uint32_t)(2 * c + 1) ^ sw7) << 4;
+            sts128(am + u0, mw[0], mw[1], mw[2], mw[3]);
+            sts128(am + u1, mw[4], mw[5], mw[6], mw[7]);
+            sts128(ac + u0, pw[0], pw[1], pw[2], pw[3]);
+            sts128(ac + u1, pw[4], pw[5], pw[6], pw[7]);
+            sts32(sfa + c * SF_TILE_BYTES, sw & 0x3F3F3F3Fu);
+          }
+        }
+        fence_async_smem();
+        mbar_arrive(bar_afull + 8 * cur.astage);
+      }
+
+      if (!seg_last) continue;
+      // ---------------- epilogue of the segment that ends with this item ----------------
+      const int tile_begin = tile * spt;
+      const int seg_begin = it_begin > tile_begin ? it_begin : tile_begin;
+      const bool complete = (seg_begin == tile_begin) && (step == spt - 1);
+      const int rt = tile / a.token_tiles, tt = tile - rt * a.token_tiles;
+      const int n_out = rt * TILE_ROWS + row;
+      const int m0 = tt * NT;
+      if (!dep_waited) {
+        grid_dep_wait();
+        if (a.extra_scale) ts *= *a.extra_scale;
+        dep_waited = true;
+      }
+      if (!wait_all(bar_accfull, seg & 1u, 27)) break;
+      tc_fence_after();
+      const int slot_idx = (seg_begin == it_begin) ? 0 : 1;
+      float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(NT * TILE_ROWS);
+#pragma unroll 1
+      for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
+        uint32_t v[16];
+        tc_ld16(tmem_base + lane_off + c0, v);
+        tc_wait_ld();
+        if (complete) {
+          if (n_out < a.g.N) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int m = m0 + c0 + j;
+              if (m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * __uint_as_float(v[j]));
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (m0 + c0 + j < a.M) my_slot[(c0 + j) * TILE_ROWS + row] = __uint_as_float(v[j]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_accempty);
+      ++seg;
+      if (complete) continue;
+      // ---------------- partial tile: publish, count, last arrival reduces ----------------
+      if (!epi_sync()) break;
+      const int tile_end = tile_begin + spt;
+      const int c_first = cta_of_item(tile_begin, grid, a.total_items);
+      const int c_last = cta_of_item(tile_end - 1, grid, a.total_items);
+      if (leader) {
+        const uint32_t parts = (uint32_t)(c_last - c_first + 1);
+        uint32_t prev;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.counters + tile) : "memory");
+        const uint32_t last = (prev + 1 == parts) ? 1u : 0u;
+        if (last) a.counters[tile] = 0;                               // leave the counter ready for the next call
+        *bcast = last;
+      }
+      if (!epi_sync()) break;
+      const bool finisher = *reinterpret_cast<volatile uint32_t*>(bcast) != 0;
+      if (!epi_sync()) break;                                         // bcast may be rewritten after this
+      if (!finisher) continue;
+#pragma unroll 1
+      for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
+        float acc[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
+        const int m_valid = a.M - (m0 + c0);
+        for (int c = c_first; c <= c_last; ++c) {                      // ascending CTA order: a fixed summation order
+          const long long b_c = (a.total_items * c) / grid;
+          const int sl = (b_c / spt == tile) ? 0 : 1;
+          const float* src = a.slots + ((size_t)c * 2 + sl) * (size_t)(NT * TILE_ROWS);
+          float part[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) part[j] = (j < m_valid) ? __ldcg(src + (c0 + j) * TILE_ROWS + row) : 0.0f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) acc[j] += part[j];
+        }
+        if (n_out < a.g.N) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            if (m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * acc[j]);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// Activation operand for the kernel above.  codes_out: [M][KP / 8] 32-bit words (KP = K rounded up to whole
+// stages, zero beyond K), each word's nibbles in the packed form's order (nibbles p and p + 4 = elements 2p and
+// 2p + 1).  sfb: [token tile][stage][chunk] tiles of 128 words; word 4 * (t % 32) + t / 32 of a tile holds the
+// four 7-bit scale bytes of token t of the tile for the chunk's four blocks (zero for tokens beyond M and
+// blocks beyond K).
+__global__ void fp4_act_prep_kernel(const uint32_t* __restrict__ codes, const uint8_t* __restrict__ scales, int M, int K,
+                                    int KP, int token_tiles, int spt, uint32_t* __restrict__ codes_out,
+                                    uint32_t* __restrict__ sfb) {
+  grid_dep_launch();
+  grid_dep_wait();
+  const long long row_words = KP / 8, in_words = K / 8;
+  const long long n_code = (long long)M * row_words;
+  const long long n_sf = (long long)token_tiles * spt * CH * 128;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_code + n_sf;
+       i += (long long)gridDim.x * blockDim.x) {
+    if (i < n_code) {
+      const long long m = i / row_words, wi = i - m * row_words;
+      const uint32_t w = wi < in_words ? codes[m * in_words + wi] : 0u;
+      uint32_t o = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o |= ((w >> (4 * j)) & 0xFu) << (4 * ((j >> 1) + 4 * (j & 1)));
+      codes_out[i] = o;
+    } else {
+      const long long s = i - n_code;
+      const int wi = (int)(s & 127);
+      const long long tile = s >> 7;                                   // (token tile, stage, chunk)
+      const int c = (int)(tile % CH);
+      const int step = (int)((tile / CH) % spt);
+      const int tt = (int)(tile / ((long long)CH * spt));
+      const int token = tt * NT + (wi >> 2) + 32 * (wi & 3);
+      const int kb0 = (step * CH + c) * 4;
+      uint32_t v = 0;
+      if (token < M) {
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb)
+          if ((kb0 + kb) * 16 < K) v |= (uint32_t)(scales[(size_t)token * (K / 16) + kb0 + kb] & 0x7Fu) << (8 * kb);
+      }
+      sfb[s] = v;
+    }
+  }
+}
+
+struct Plan {
+  int token_tiles, steps_per_tile, grid, KP;
+  long long tiles, total_items;
+  size_t counters_bytes, slots_bytes, codes_bytes, sfb_bytes;
+};
+
+static Plan make_plan(const razer_desc* d, int M) {
+  Plan p;
+  const Geometry g = make_geometry(d->N, d->K);
+  p.token_tiles = (M + NT - 1) / NT;
+  p.steps_per_tile = (g.k_chunks + CH - 1) / CH;
+  p.KP = p.steps_per_tile * CH * CHUNK_K;
+  p.tiles = (long long)g.row_tiles * p.token_tiles;
+  p.total_items = p.tiles * p.steps_per_tile;
+  const int sms = sm_count();
+  p.grid = (int)(p.total_items < sms ? p.total_items : sms);
+  p.counters_bytes = align256((size_t)p.tiles * sizeof(uint32_t));
+  p.slots_bytes = (size_t)(p.grid > 148 ? p.grid : 148) * 2 * NT * TILE_ROWS * sizeof(float);
+  p.codes_bytes = align256((size_t)M * p.KP / 2);
+  p.sfb_bytes = (size_t)p.token_tiles * p.steps_per_tile * SF_BYTES;
+  return p;
+}
+
+// FP4 magnitude code (0 .5 1 1.5 2 3 4 6 -> 0..7) of v, or -1.
+static int fp4_code_of(float v) {
+  const float mags[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+  for (int i = 1; i < 8; ++i)
+    if (mags[i] == v) return i;
+  return -1;
+}
+
+// Base / remainder pair of each special-value magnitude (App. D.3): the largest base that serves both
+// magnitudes when there is one (4 for {5, 8}: 4 + 1 and 4 + 4), otherwise each magnitude's own largest base.
+static bool split_special_values(const float sv[2], uint32_t base[2], uint32_t rem[2]) {
+  const float mags[7] = {6.0f, 4.0f, 3.0f, 2.0f, 1.5f, 1.0f, 0.5f};   // descending
+  for (int bi = 0; bi < 7; ++bi) {                                     // a base that serves both magnitudes
+    const int r0 = fp4_code_of(sv[0] - mags[bi]), r1 = fp4_code_of(sv[1] - mags[bi]);
+    if (r0 > 0 && r1 > 0) {
+      base[0] = base[1] = (uint32_t)fp4_code_of(mags[bi]);
+      rem[0] = (uint32_t)r0;
+      rem[1] = (uint32_t)r1;
+      return true;
+    }
+  }
+  for (int s = 0; s < 2; ++s) {                                        // each magnitude on its own
+    bool found = false;
+    for (int bi = 0; bi < 7 && !found; ++bi) {
+      const int r = fp4_code_of(sv[s] - mags[bi]);
+      if (r > 0) {
+        base[s] = (uint32_t)fp4_code_of(mags[bi]);
+        rem[s] = (uint32_t)r;
+        found = true;
+      }
+    }
+    if (!found) return false;
+  }
+  return true;
+}
+
+}  // namespace fp4_path
+
+size_t gemm_fp4_workspace_bytes(const razer_desc* d, int M) {
+  const fp4_path::Plan p = fp4_path::make_plan(d, M);
+  return WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes + p.codes_bytes + p.sfb_bytes;
+}
+
+int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_codes, const uint8_t* act_scales,
+                    const float* act_tensor_scale_dev, int M, void* y, void* ws, size_t ws_bytes, cudaStream_t st) {
+  using namespace fp4_path;
+  const Geometry g = make_geometry(d->N, d->K);
+  const Plan p = make_plan(d, M);
+  const size_t need = gemm_fp4_workspace_bytes(d, M);
+  if (!ws || ws_bytes < need)
+    return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+  Args a;
+  {
+    uint32_t base[2], rem[2];
+    if (!split_special_values(d->sv_mag, base, rem))
+      return set_error(RAZER_ERR_UNSUPPORTED, "special values %g / %g are not sums of two FP4 values", d->sv_mag[0],
+                       d->sv_mag[1]);
+    a.base0 = base[0];
+    a.rem0 = rem[0];
+    a.base1 = base[1];
+    a.rem1 = rem[1];
+  }
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  char* base_ws = (char*)ws;
+  a.status = (uint32_t*)base_ws;
+  a.counters = (uint32_t*)(base_ws + WS_STATUS_BYTES);
+  a.slots = (float*)(base_ws + WS_STATUS_BYTES + p.counters_bytes);
+  uint8_t* codes_pad = (uint8_t*)(base_ws + WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes);
+  uint8_t* sfb = codes_pad + p.codes_bytes;
+  a.sfb = sfb;
+  a.y = (__nv_bfloat16*)y;
+  a.extra_scale = act_tensor_scale_dev;
+  a.g = g;
+  a.tensor_scale = d->tensor_scale;
+  a.M = M;
+  a.token_tiles = p.token_tiles;
+  a.steps_per_tile = p.steps_per_tile;
+  a.total_items = p.total_items;
+
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUtensorMap tmap_x, tmap_w;
+  {
+    // padded activation codes as bytes: [M][KP / 2]; box = 128 bytes (one stage of k) x NT tokens
+    const cuuint64_t dims[2] = {(cuuint64_t)(p.KP / 2), (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)(p.KP / 2)};
+    const cuuint32_t box[2] = {128, (cuuint32_t)NT};
+    const CUresult r = enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, codes_pad, dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled (activation codes) failed with code %d", (int)r);
+  }
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)(PIECE_BYTES / 8), (cuuint64_t)g.k_chunks, (cuuint64_t)g.strips()};
+    const cuuint64_t strides[2] = {(cuuint64_t)PIECE_BYTES, (cuuint64_t)g.strip_bytes()};
+    const cuuint32_t box[3] = {(cuuint32_t)(PIECE_BYTES / 8), (cuuint32_t)CH, (cuuint32_t)TILE_STRIPS};
+    const CUresult r = enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_INT64, 3, const_cast<void*>(packed), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(RAZER_ERR_CUDA, "cuTensorMapEncodeTiled (weights) failed with code %d", (int)r);
+  }
+  static const bool pdl = [] { const char* e = getenv("RAZER_PDL"); return !(e && e[0] == '0'); }();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  {
+    const long long work = (long long)M * (p.KP / 8) + (long long)p.token_tiles * p.steps_per_tile * CH * 128;
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, fp4_act_prep_kernel, (const uint32_t*)act_codes, act_scales, M, d->K, p.KP,
+                                             p.token_tiles, p.steps_per_tile, (uint32_t*)codes_pad, (uint32_t*)sfb);
+    count_launches(1);
+    RAZER_TRY(check_cuda(e, "fp4_act_prep_kernel launch"));
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    RAZER_TRY(check_cuda(cudaFuncSetAttribute(razer_fp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES),
+                         "cudaFuncSetAttribute(max dynamic shared memory)"));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, razer_fp4_kernel, tmap_x, tmap_w, a);
+  count_launches(1);
+  return check_cuda(e, "razer_fp4_kernel launch");
+}
+
+}  // namespace razer

@@ -67,4 +67,5 @@ def test_host_side_validation(binding):
     assert b.lib().razer_gemv(ctypes.byref(good), 24, 16, 1, 16, None, 0, None) == b.ERR_INVALID_ARG  # packed misaligned
     assert b.lib().razer_quant_act(None, 4, 64, 5.0, None, None, None, None, None, None) == b.ERR_INVALID_ARG
     assert b.lib().razer_quant_act(16, 4, 72, 5.0, None, None, None, None, None, None) == b.ERR_INVALID_ARG
-    assert b.lib().razer_gemm_w4a4(ctypes.byref(good), 16, 16, 16, 16, 5.0, 4, 16, 256, 1 << 20, 1, None) == b.ERR_UNSUPPORTED
+    # the block-scaled FP4 path checks its workspace before it launches anything
+    assert b.lib().razer_gemm_w4a4(ctypes.byref(good), 16, 16, 16, 16, 5.0, 4, 16, 256, 1 << 10, 1, None) == b.ERR_WORKSPACE

@@ -334,6 +334,95 @@ def test_w4a4_oracle_quantized(b, M, N, K):
     assert err <= TOL, f"relative Frobenius error {err:.3e}"
 
 
+def _w4a4_native_check(b, desc, packed, wc, ws, wd, ac, as_, ats, rows=None, **kw):
+    """Two-pass block-scaled FP4 path against the oracle's W4A4 matmul: relative Frobenius bar and the
+    element-wise bound of the other matmul kernels (FP32 accumulation of exact products)."""
+    M = ac.shape[0]
+    wsb = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+    y = b.razer_gemm_w4a4(desc, packed, ac, as_, ats, workspace=wsb, use_native_fp4=True)
+    b.razer_workspace_status(wsb)
+    y2 = b.razer_gemm_w4a4(desc, packed, ac, as_, ats, workspace=wsb, use_native_fp4=True)
+    b.razer_workspace_status(wsb)
+    assert torch.equal(y, y2), "second call with the same workspace differs"
+    acn, asn = ac.cpu().numpy(), as_.cpu().numpy()
+    if rows is not None:
+        wc, ws, y = wc[rows], ws[rows], y[:, torch.from_numpy(rows).cuda()]
+    da = ro.dequant_d1(acn, asn, scale_fmt=ro.SCALE_E4M3_META1, sv_mag=(5.0, 5.0)).astype(np.float64)
+    dw = ro.dequant_d1(wc, ws, **kw).astype(np.float64)
+    scale = float(np.float32(wd)) * float(np.float32(ats.item()))
+    y64 = scale * (da @ dw.T)
+    mag = abs(scale) * (np.abs(da) @ np.abs(dw).T)
+    ref = ro.f64_to_bf16_bits(y64)
+    if kw.get("remap_code", 0x8) == 0x8:            # (the oracle's W4A4 matmul takes one remapped code for both operands)
+        assert np.array_equal(ref, ro.matmul_w4a4(acn, asn, np.float32(ats.item()), wc, ws, np.float32(wd),
+                                                  sv_mag_w=kw.get("sv_mag", (5.0, 8.0))))
+    err = rel_fro_bits(y, ref)
+    bad, differ, total = elementwise_report(y, ref, y64, mag)
+    print(f"[parity] native FP4 {tuple(ac.shape)} x {tuple(wc.shape)}: rel fro {err:.2e}, {differ} of {total} differ, {bad} out of bound")
+    assert err <= TOL and bad == 0
+
+
+@pytest.mark.parametrize("M,N,K,sv_mag,remap_code", [(256, 512, 8192, (5.0, 8.0), 0x8), (17, 200, 464, (5.0, 8.0), 0x8),
+                                                    (130, 300, 2048, (2.5, 12.0), 0x0), (13, 520, 1040, (7.0, 10.0), 0x8),
+                                                    (300, 260, 272, (5.0, 8.0), 0x8)])
+def test_w4a4_native_fp4_two_pass(b, M, N, K, sv_mag, remap_code):
+    """App. D.3: RaZeR weights as B_main + B_comp on the block-scaled FP4 tensor-core path, activations in plain
+    NVFP4 (quantized on the GPU with no special value, checked against the oracle's Eq. 1-3)."""
+    w = inputs.student_t_weights(N, K, 300 + M, outlier_frac=0.001).numpy()
+    wc, ws, wd = ro.quantize_weight(w, sv_mag=sv_mag, remap_code=remap_code)
+    desc = b.make_desc(N, K, float(wd), sv_mag=sv_mag, remap_code=remap_code)
+    packed = b.razer_pack_layout(desc, torch.from_numpy(wc).cuda(), torch.from_numpy(ws).cuda())
+    x = inputs.activations(M, K, 301, outlier_channel_frac=0.01)
+    ac, as_, ats = b.razer_quant_act(x.cuda(), sv_mag=0.0)
+    torch.cuda.synchronize()
+    want_c, want_s, want_d = ro.quantize_act(inputs.bf16_to_bits(x), sv_mag=None)
+    assert np.float32(ats.item()) == want_d
+    assert np.array_equal(ac.cpu().numpy(), want_c) and np.array_equal(as_.cpu().numpy(), want_s)
+    _w4a4_native_check(b, desc, packed, wc, ws, wd, ac, as_, ats, sv_mag=sv_mag, remap_code=remap_code)
+
+
+def test_w4a4_native_fp4_decodes_bit_exactly(b):
+    """One-hot NVFP4 activations (code 1.0, block scale 1.0) through the two-pass path: y[m, n] is the tensor
+    scale times one decoded weight, exact whatever the accumulation order, so main + comp is checked bit for bit."""
+    N, K, TS = 300, 1104, 0.25
+    for remap_code, sv_mag, seed in [(0x8, (5.0, 8.0), 211), (0x0, (2.5, 12.0), 212)]:
+        codes, scales = inputs.random_codes(N, K, seed=seed, scale_lo=0, scale_hi=64, zero_block_frac=0.05)
+        codes, scales = codes.numpy(), scales.numpy()
+        want = ro.dequant_d1(codes, scales, sv_mag=sv_mag, remap_code=remap_code).astype(np.float64) * TS
+        want_bits = ro.f64_to_bf16_bits(want)
+        desc = b.make_desc(N, K, TS, sv_mag=sv_mag, remap_code=remap_code)
+        packed = b.razer_pack_layout(desc, torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda())
+        M = 160                                                        # two token tiles, the second ragged
+        wsb = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+        one = torch.ones(1, dtype=torch.float32, device="cuda")
+        got = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+        as_ = torch.full((M, K // 16), 0x38, dtype=torch.uint8, device="cuda")      # E4M3 1.0 everywhere
+        ar = torch.arange(M, device="cuda")
+        for k0 in range(0, K, M):
+            m = min(M, K - k0)
+            ac = torch.zeros((M, K // 2), dtype=torch.uint8, device="cuda")
+            kk = k0 + ar[:m]
+            ac[ar[:m], kk // 2] = torch.where(kk % 2 == 0, 0x02, 0x20).to(torch.uint8)   # FP4 code of 1.0
+            y = b.razer_gemm_w4a4(desc, packed, ac, as_, one, workspace=wsb, use_native_fp4=True)
+            got[:, k0:k0 + m] = y[:m].t()
+        b.razer_workspace_status(wsb)
+        got_bits = inputs.bf16_to_bits(got.cpu())
+        g = np.where((got_bits & 0x7FFF) == 0, 0, got_bits)
+        wv = np.where((want_bits & 0x7FFF) == 0, 0, want_bits)
+        bad = np.argwhere(g != wv)
+        assert bad.size == 0, (remap_code, sv_mag, len(bad), bad[:5].tolist())
+
+
+def test_w4a4_native_fp4_config5_full_size_sampled_rows(b):
+    M, N, K = 256, 8192, 8192
+    wc, ws = inputs.random_codes(N, K, seed=97)
+    wc, ws = wc.numpy(), ws.numpy()
+    desc, packed = _pack(b, wc, ws, 0.002)
+    x = inputs.activations(M, K, 97, outlier_channel_frac=0.01)
+    ac, as_, ats = b.razer_quant_act(x.cuda(), sv_mag=0.0)
+    _w4a4_native_check(b, desc, packed, wc, ws, 0.002, ac, as_, ats, rows=sample_rows(N, 128, 98))
+
+
 def test_w4a4_config5_full_size_sampled_rows(b):
     M, N, K = 256, 8192, 8192
     wc, ws = inputs.random_codes(N, K, seed=95)

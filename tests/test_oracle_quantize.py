@@ -344,3 +344,32 @@ def test_scale_aware_brute_force_over_its_candidates_on_tiny_blocks():
                     e = (vals[:, None] - wb[r, b][None, :]) ** 2       # [16 values, 2 elements]
                     best = min(best, e[:, 0].min() + e[:, 1].min())
             assert got[r, b] <= best * (1 + 1e-4) + 1e-18      # midpoint decisions are taken on FP32-rounded xs
+
+
+# --------------------------------------------------------------------------
+# plain NVFP4 (Sec. 3, Eq. 1-3): the activation format of the two-pass realization (App. D.3)
+# --------------------------------------------------------------------------
+
+def test_plain_nvfp4_is_eq_1_to_3_alone():
+    x = inputs.activations(6, 512, 31, outlier_channel_frac=0.02)
+    xb = inputs.bf16_to_bits(x)
+    c, s, d32, dbg = ro.quantize_act(xb, sv_mag=None, return_debug=True)
+    # no special-value code, no metadata bit; decoding it as RaZeR or as NVFP4 is the same thing
+    nib = ro.unpack_codes(c)
+    assert not np.any(nib == 0x8) and not np.any(s & 0x80)
+    xf = ro.bf16_bits_to_f32(xb).astype(np.float64)
+    # Eq. 3 by brute force: every element is the nearest point of the FP4 grid to xs (ties aside)
+    grid = np.array(sorted({ro.fp4_value(k) for k in range(16)}))
+    xs = dbg["xs"].astype(np.float64).reshape(6, 512)
+    q, sv = ro.decode_block_values(c, s, scale_fmt=ro.SCALE_E4M3_META1, sv_mag=(5.0, 5.0))
+    nearest = np.abs(xs[..., None] - grid).min(axis=-1)
+    assert np.all(np.abs(xs - q) <= nearest + 1e-6)
+    # Eq. 6's invariant: adding a special value never raises a block's error at the same scale
+    c2, s2, d2, dbg2 = ro.quantize_act(xb, sv_mag=(5.0,), return_debug=True)
+    assert d2 == d32 and np.array_equal(s & 0x7F, s2 & 0x7F)
+    assert np.all(dbg2["errs64"].min(axis=0) <= dbg["err_fp4"] + 1e-12)
+    # re-quantizing the dequantized tensor with the same tensor scale returns the same codes
+    d2v = ro.dequant_d2(c, s, d32, scale_fmt=ro.SCALE_E4M3_META1, sv_mag=(5.0, 5.0)).astype(np.float32)
+    c3, s3, _ = ro.quantize(d2v, ro.SCALE_E4M3_META1, None, tensor_scale=d32)
+    assert np.array_equal(c3, c) and np.array_equal(s3, s)
+    assert np.linalg.norm(d2v - xf) / np.linalg.norm(xf) < 0.12
