@@ -34,8 +34,8 @@ DECODE_SHAPES = [(4096, 4096), (11008, 4096), (4096, 11008)]
 SKINNY_SHAPES = [(8192, 8192), (28672, 8192), (8192, 28672)]
 PREFILL_SHAPES = [(14336, 4096), (4096, 14336)]
 # DRAM bytes of one step (its three launches) read from the ncu capture of the kernel as committed:
-# 9,465,344 + 25,390,592 + 25,404,416 read, 0 written.  Set to None whenever the kernel changes until re-captured.
-NCU_DRAM_BYTES_PER_STEP = 60260352
+# 9,506,304 + 25,430,272 + 25,445,120 read, 0 written.  Set to None whenever the kernel changes until re-captured.
+NCU_DRAM_BYTES_PER_STEP = 60381696
 METRIC = "razer_gemv_effective_hbm_bandwidth"
 
 
@@ -353,8 +353,8 @@ def main():
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": pk["hbm"], "unit": "GB/s",
                      "frac": value / world / pk["hbm"], "traffic": NCU_DRAM_BYTES_PER_STEP, "peak_source": pk["source"],
                      "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the step's three launches "
-                                       "(profiles/razer_direct_kernel_gemv_config2.md)",
-                     "kernel": "razer_gemv (3 launches per step)", "algorithmic_bytes_per_step": step_bytes,
+                                       "(profiles/razer_stream_kernel_gemv_config2.md)",
+                     "kernel": "razer_stream_kernel via razer_gemv (3 launches per step)", "algorithmic_bytes_per_step": step_bytes,
                      "frac_of_nominal_8TBps": value / world / 8000.0},
         "decode_per_shape": per_shape,
     }
@@ -410,6 +410,18 @@ def main():
         tf = 2.0 * M * N * K / (t * 1e-3) / 1e12
         extras.append({"config": 5, "op": "razer_gemm_w4a4", "M": M, "N": N, "K": K, "us": t * 1e3, "TFLOPs": tf,
                        "frac_bf16": tf / pk["bf16"]})
+        # the two-pass block-scaled FP4 realization (RaZeR weights x plain-NVFP4 activations); operations counted
+        # as 2MNK although two passes execute; the FP4 peak is the measured bf16 peak x the nominal ratio of 4
+        ac0, as0, ats0 = b.razer_quant_act(x, sv_mag=0.0)
+        ws4 = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")       # a workspace serves one of the two paths
+        f4 = lambda i: b.razer_gemm_w4a4(desc, sets[i % 4], ac0, as0, ats0, y=y, workspace=ws4, use_native_fp4=True)
+        for i in range(3):
+            f4(i)
+        t4 = graph_time(f4, 8)
+        tf4 = 2.0 * M * N * K / (t4 * 1e-3) / 1e12
+        extras.append({"config": 5, "op": "razer_gemm_w4a4 (two-pass block-scaled FP4)", "M": M, "N": N, "K": K,
+                       "us": t4 * 1e3, "TFLOPs_effective": tf4, "frac_fp4_two_pass": 2.0 * tf4 / (4.0 * pk["bf16"]),
+                       "GBps": algo_bytes(M, N, K) / (t4 * 1e-3) / 1e9, "frac_hbm": algo_bytes(M, N, K) / (t4 * 1e-3) / 1e9 / pk["hbm"]})
         # GPU weight quantizer (offline step; FP32 in, interchange format out), 4096 x 4096
         wq = inputs.student_t_weights(4096, 4096, 5000, outlier_frac=0.001).cuda()
         b.razer_quant_weight(wq)

@@ -209,7 +209,8 @@ int razer_decode_act(const uint8_t* act_codes_dev, const uint8_t* act_scales_dev
  * y = bf16( w_scale * a_scale * sum_k decoded_act[m][k] * decoded_w[n][k] ).
  * act_codes_dev [M][K/2], act_scales_dev [M][K/16], act_tensor_scale_dev: one device float, as
  * razer_quant_act writes them.  The workspace (RAZER_OP_GEMM_W4A4, zeroed once by
- * razer_workspace_init, 256-byte aligned) serves either path below.
+ * razer_workspace_init, 256-byte aligned) is large enough for either path below, but the two
+ * lay it out differently: zero it again before a call that takes the other path.
  * use_native_fp4 = 0: both operands RaZeR; the activations are decoded to bf16 (exact) into the
  * workspace and multiplied by the bf16 tensor-core kernel of razer_gemm.
  * use_native_fp4 != 0: the two-pass realization of App. D.3 on the block-scaled FP4 tensor-core

@@ -12,8 +12,8 @@
 // Mapping: the weight tile is the MMA's A operand (128 rows), the token tile its B operand (128 tokens),
 // both K-major FP4 in shared memory with the 128-byte swizzle (one row = 256 codes = one stage of four
 // chunks).  Warp 0 = TMA producer (packed weights, activation codes, activation scale factors), warp 1 =
-// TMEM owner and MMA issuer, warps 2..9 = remap (thread = weight row; two groups of four warps take the
-// stages in turn) and epilogue.  A remap thread reads its row's packed blocks, finds the special-value
+// TMEM owner and MMA issuer, warps 2..17 = remap (thread = weight row and half of a stage's chunks; two groups of eight warps take
+// the stages in turn) and epilogue.  A remap thread reads its row's packed blocks, finds the special-value
 // nibbles (the only nibbles that are 0x0 in the packed form), builds the two code words with two integer
 // multiply-adds, applies the block's stored-negated flag to the sign bits, and writes both rows plus the row's
 // four scale bytes (scale-factor layout: 32 x 16-byte rows, row r % 32, word r / 32).  The MMA warp copies
@@ -40,7 +40,7 @@ constexpr int NT = 128;                               // tokens per tile (MMA N)
 constexpr int CH = 4;                                 // chunks per stage: 256 codes = one 128-byte swizzled row
 constexpr int STAGES = 4;                             // shared-memory ring fed by TMA
 constexpr int ASTAGES = 2;                            // remapped-operand ring, one slot per remap group
-constexpr int NRW = 8;                                // remap warps
+constexpr int NRW = 16;                               // remap warps: two groups of eight
 constexpr int THREADS = 64 + 32 * NRW;
 constexpr int W_BYTES = CH * CHUNK_BYTES;             // 18432 packed weight bytes of a stage
 constexpr int X_BYTES = NT * 128;                     // activation codes of a stage
@@ -50,9 +50,10 @@ constexpr int STAGE_BYTES = W_BYTES + X_BYTES + SF_BYTES;
 constexpr int A_TILE_BYTES = TILE_ROWS * 128;         // 128 rows x 256 codes
 constexpr int ASTAGE_BYTES = 2 * A_TILE_BYTES + SF_BYTES;
 constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 4;
-constexpr int ACC_COLS = NT;
+constexpr int NACC = 2;                               // accumulators: the main pass adds into one, the comp pass into the other
+constexpr int ACC_COLS = NACC * NT;
 constexpr int SF_COLS = 2 * CH * 4;                   // per operand ring slot: A and B scale factors of four chunks
-constexpr int TMEM_COLS = 256;
+constexpr int TMEM_COLS = 512;
 constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + (size_t)ASTAGES * ASTAGE_BYTES + NUM_BARS * 8 + 64;
 static_assert(STAGE_BYTES % 1024 == 0 && W_BYTES % 1024 == 0 && ASTAGE_BYTES % 1024 == 0, "swizzled tiles sit on 1024 bytes");
 static_assert(ACC_COLS + ASTAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
@@ -146,7 +147,7 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       mbar_init(bar_empty + 8 * i, 1);
     }
     for (int i = 0; i < ASTAGES; ++i) {
-      mbar_init(bar_afull + 8 * i, 128);
+      mbar_init(bar_afull + 8 * i, 256);
       mbar_init(bar_aempty + 8 * i, 1);
     }
     mbar_init(bar_accfull, 1);
@@ -247,17 +248,25 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       const uint32_t sfa_s = am + 2 * A_TILE_BYTES;
       const uint32_t sf_t = tmem_sf0 + cur.astage * SF_COLS;
       if (elect_one()) {
+        // the stage's scale factors first, then its MMAs back to back
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+          if (c < nch) {
+            copy_sf_to_tmem(sf_t + c * 4, sfa_s + c * SF_TILE_BYTES);
+            copy_sf_to_tmem(sf_t + CH * 4 + c * 4, sfb_s + c * SF_TILE_BYTES);
+          }
+        }
+        // Main and comp passes add into accumulators of their own (summed in the epilogue): MMAs on one
+        // accumulator execute one after the other, and consecutive MMAs then never share one.
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           if (c < nch) {
             const uint32_t sfa_t = sf_t + c * 4, sfb_t = sf_t + CH * 4 + c * 4;
-            copy_sf_to_tmem(sfa_t, sfa_s + c * SF_TILE_BYTES);
-            copy_sf_to_tmem(sfb_t, sfb_s + c * SF_TILE_BYTES);
             // 64 codes further along k: +32 bytes inside the 128-byte rows
             const uint32_t b_lo = ((xs + c * 32) >> 4) | (1u << 16);
-            mma_fp4(tmem_base, ((am + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t,
-                    (seg_first && c == 0) ? 0u : 1u);
-            mma_fp4(tmem_base, ((ac + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t, 1u);
+            const uint32_t acc = (seg_first && c == 0) ? 0u : 1u;
+            mma_fp4(tmem_base, ((am + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t, acc);
+            mma_fp4(tmem_base + NT, ((ac + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t, acc);
           }
         }
         tc_commit(bar_empty + 8 * cur.stage);
@@ -278,11 +287,15 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // ===================== remap (thread = weight row) + epilogue =====================
     const int row = 32 * (warp & 3) + lane;              // weight row of the tile = TMEM lane of its outputs
     const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
-    const int group = (warp - 2) >> 2;
-    constexpr int GROUPS = NRW / 4;
+    // Eight warps remap one item together: warps w and w + 4 of a group own the same 32 rows (a warp reaches only
+    // the TMEM lanes 32 * (warp % 4) .. + 31, which the epilogue needs) and take two of the stage's four chunks each.
+    const int group = (warp - 2) >> 3;
+    const int half = ((warp - 2) >> 2) & 1;
+    constexpr int GROUPS = NRW / 8;
     static_assert(GROUPS == ASTAGES && STAGES >= ASTAGES, "an operand slot per group; see the wait order below");
-    const int col_lo = 16 * ((group * (NT / 16)) / GROUPS);
-    const int col_hi = 16 * (((group + 1) * (NT / 16)) / GROUPS);
+    constexpr int EPI_SETS = NRW / 4;                     // sets of four warps (all lane quarters) share the columns
+    const int col_lo = 16 * ((((warp - 2) >> 2) * (NT / 16)) / EPI_SETS);
+    const int col_hi = 16 * (((((warp - 2) >> 2) + 1) * (NT / 16)) / EPI_SETS);
     const bool leader = (threadIdx.x == 64);
     float ts = a.tensor_scale;
     bool dep_waited = false;
@@ -324,7 +337,8 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const uint32_t ac = am + A_TILE_BYTES;
         const uint32_t sfa = smem_addr(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES + 2 * A_TILE_BYTES + sf_word;
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
+        for (int cc = 0; cc < CH / 2; ++cc) {
+          const int c = half * (CH / 2) + cc;
           if (c < nch) {
             const uint32_t ck = st + c * PIECE_BYTES;
             const uint2 sq = lds64(ck + scale_off);
@@ -379,9 +393,12 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(NT * TILE_ROWS);
 #pragma unroll 1
       for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
-        uint32_t v[16];
+        uint32_t v[16], v1[16];
         tc_ld16(tmem_base + lane_off + c0, v);
+        tc_ld16(tmem_base + lane_off + NT + c0, v1);
         tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v1[j]));
         if (complete) {
           if (n_out < a.g.N) {
 #pragma unroll
