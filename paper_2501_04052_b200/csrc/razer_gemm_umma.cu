@@ -21,9 +21,11 @@
 // several output tiles, partial results reduced through global memory): the grid is
 // persistent, work items are (output tile, k-stage) pairs in tile-major order and every CTA
 // takes one contiguous stripe of items.  A stripe's first and last tile may be partial; those
-// go to a per-CTA FP32 slot in the workspace and the last CTA to arrive at a tile (one
-// counter per tile) adds the slots in CTA order, scales and rounds once.  Tiles a stripe
-// covers completely are written directly.
+// go to a per-CTA FP32 slot in the workspace.  The CTA that holds a tile's first items (its
+// stripe ends inside the tile) owns the tile: it waits until the other CTAs of the tile have
+// counted themselves in (one counter per tile; for them the tile came first, so they are
+// long done), adds the slots in CTA order, scales and rounds once.  Tiles a stripe covers
+// completely are written directly.
 //
 // Every wait (mbarrier, counter) is bounded: on expiry the thread records a code in the
 // workspace status word and the kernel drains and exits instead of hanging the GPU.
@@ -440,10 +442,30 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         if (a.extra_scale) ts *= *a.extra_scale;
         dep_waited = true;
       }
+      // A partial tile is finished by its owner, the CTA whose stripe holds the tile's FIRST items: for that CTA the
+      // tile is the end of its stripe, for every other CTA of the tile it is the beginning, so their parts were
+      // published (FP32 slot in the workspace, then a release-add on the tile's counter) long before the owner gets
+      // here.  The owner adds its own accumulator (straight from TMEM) and the other parts in CTA order.
+      const int c_first = cta_of_item(tile_begin, grid, a.total_items);
+      const int c_last = cta_of_item(tile_begin + spt - 1, grid, a.total_items);
+      const bool owner = !complete && cta == c_first;
+      if (owner) {
+        // acquire: every counted CTA's slot stores are visible to this thread's loads below
+        const uint32_t others = (uint32_t)(c_last - c_first);
+        uint32_t seen = 0;
+        const uint64_t t0 = global_ns();
+        for (;;) {
+          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters + tile) : "memory");
+          if (seen >= others || *abort_flag || global_ns() - t0 > WAIT_LIMIT_NS) break;
+          __nanosleep(200);
+        }
+        const bool ready = seen >= others;
+        if (!ready) fail(9);
+        if (!__all_sync(0xFFFFFFFFu, ready)) break;
+      }
       if (!wait_all(bar_accfull, seg & 1u, 7)) break;
       tc_fence_after();
-      const int slot_idx = (seg_begin == it_begin) ? 0 : 1;          // first segment of the stripe or not
-      float* my_slot = a.slots + ((size_t)cta * 2 + slot_idx) * (size_t)(NT * TILE_ROWS);
+      float* my_slot = a.slots + (size_t)cta * 2 * (size_t)(NT * TILE_ROWS);   // a non-owner's part is its stripe's first segment
       bool acc_valid[GROUPS];                                         // GI: which groups had an item in this segment
       {
         const int i0 = seg_begin - it_begin, len = i - i0 + 1;
@@ -469,7 +491,26 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
           }
         }
-        if (complete) {
+        if (complete || owner) {
+          if (owner) {
+            const int m_valid = a.M - (m0 + c0);                       // tokens of this column group that exist
+            // ascending CTA order (a fixed summation order); the loads of two CTAs' slots are in flight together
+            for (int cb = c_first + 1; cb <= c_last; cb += 2) {
+              float part[2][16];
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {
+                const int c = cb + u <= c_last ? cb + u : c_last;
+                const float* src = a.slots + (size_t)c * 2 * (size_t)(NT * TILE_ROWS);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  part[u][j] = (cb + u <= c_last && j < m_valid) ? __ldcg(src + (c0 + j) * TILE_ROWS + row) : 0.0f;
+              }
+#pragma unroll
+              for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + part[u][j]);
+            }
+          }
           if (n_out < a.g.N) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -487,56 +528,11 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
       mbar_arrive(bar_accempty);
       ++seg;
       if (complete) continue;
-      // ---------------- partial tile: publish, count, last arrival reduces ----------------
-      if (!epi_sync()) break;                                         // all slot stores of this CTA are done (CTA scope)
-      const int tile_end = tile_begin + spt;
-      const int c_first = cta_of_item(tile_begin, grid, a.total_items);
-      const int c_last = cta_of_item(tile_end - 1, grid, a.total_items);
+      if (!epi_sync()) break;                                         // every thread has read the counter / stored its part
       if (leader) {
-        const uint32_t parts = (uint32_t)(c_last - c_first + 1);
-        // release: the CTA's slot stores (ordered before this by the rendezvous) become visible with the count;
-        // acquire: the last arrival sees every earlier arrival's slot stores
-        uint32_t prev;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.counters + tile) : "memory");
-        const uint32_t last = (prev + 1 == parts) ? 1u : 0u;
-        if (last) a.counters[tile] = 0;                               // leave the counter ready for the next call
-        *bcast = last;
-      }
-      if (!epi_sync()) break;
-      const bool finisher = *reinterpret_cast<volatile uint32_t*>(bcast) != 0;
-      if (!epi_sync()) break;                                         // bcast may be rewritten after this
-      if (!finisher) continue;
-#pragma unroll 1
-      for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
-        float acc[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
-        const int m_valid = a.M - (m0 + c0);                           // tokens of this column group that exist
-        // ascending CTA order (a fixed summation order); the loads of two CTAs' slots are in flight together
-        for (int cb = c_first; cb <= c_last; cb += 2) {
-          float part[2][16];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int c = cb + u;
-            const long long b_c = (a.total_items * (c <= c_last ? c : c_last)) / grid;
-            const int sl = (b_c / spt == tile) ? 0 : 1;
-            const float* src = a.slots + ((size_t)(c <= c_last ? c : c_last) * 2 + sl) * (size_t)(NT * TILE_ROWS);
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              part[u][j] = (c <= c_last && j < m_valid) ? __ldcg(src + (c0 + j) * TILE_ROWS + row) : 0.0f;
-          }
-#pragma unroll
-          for (int u = 0; u < 2; ++u)
-#pragma unroll
-            for (int j = 0; j < 16; ++j) acc[j] += part[u][j];
-        }
-        if (n_out < a.g.N) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int m = m0 + c0 + j;
-            if (m < a.M) a.y[(size_t)m * a.g.N + n_out] = __float2bfloat16_rn(ts * acc[j]);
-          }
-        }
+        if (owner) a.counters[tile] = 0;                              // leave the counter ready for the next call
+        // release: the CTA's slot stores (ordered before this by the rendezvous) become visible with the count
+        else asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.counters + tile) : "memory");
       }
       (void)it;
     }
