@@ -36,32 +36,42 @@
 namespace razer {
 namespace fp4_path {
 
-constexpr int NT = 128;                               // tokens per tile (MMA N)
 constexpr int CH = 4;                                 // chunks per stage: 256 codes = one 128-byte swizzled row
-constexpr int STAGES = 4;                             // shared-memory ring fed by TMA
+constexpr int WSTAGES = 4;                            // packed-weight ring (released by the remap warps)
 constexpr int ASTAGES = 2;                            // remapped-operand ring, one slot per remap group
 constexpr int NRW = 16;                               // remap warps: two groups of eight
-constexpr int THREADS = 64 + 32 * NRW;
+constexpr int THREADS = 64 + 32 * NRW + 32;           // + W producer, MMA warp, X producer
 constexpr int W_BYTES = CH * CHUNK_BYTES;             // 18432 packed weight bytes of a stage
-constexpr int X_BYTES = NT * 128;                     // activation codes of a stage
 constexpr int SF_TILE_BYTES = 512;                    // scale factors of 128 rows x one chunk
-constexpr int SF_BYTES = CH * SF_TILE_BYTES;
-constexpr int STAGE_BYTES = W_BYTES + X_BYTES + SF_BYTES;
+constexpr int SF_BYTES = CH * SF_TILE_BYTES;          // ... x one stage
 constexpr int A_TILE_BYTES = TILE_ROWS * 128;         // 128 rows x 256 codes
 constexpr int ASTAGE_BYTES = 2 * A_TILE_BYTES + SF_BYTES;
-constexpr int NUM_BARS = 2 * STAGES + 2 * ASTAGES + 4;
-constexpr int NACC = 2;                               // accumulators: the main pass adds into one, the comp pass into the other
-constexpr int ACC_COLS = NACC * NT;
-constexpr int SF_COLS = 2 * CH * 4;                   // per operand ring slot: A and B scale factors of four chunks
-constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + (size_t)ASTAGES * ASTAGE_BYTES + NUM_BARS * 8 + 64;
-static_assert(STAGE_BYTES % 1024 == 0 && W_BYTES % 1024 == 0 && ASTAGE_BYTES % 1024 == 0, "swizzled tiles sit on 1024 bytes");
-static_assert(ACC_COLS + ASTAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
-static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+
+// NT = tokens per tile (the MMA's N): 128, or 256 when there are more than 128 tokens (half the weight traffic
+// and remap work per flop).
+template <int NT>
+struct Cfg {
+  static constexpr int XSTAGES = NT == 128 ? 3 : 2;               // activation ring (released by the MMAs' completion)
+  static constexpr int X_CODE_BYTES = NT * 128;
+  static constexpr int X_BYTES = X_CODE_BYTES + (NT / 128) * SF_BYTES;   // codes + scale-factor tiles
+  static constexpr int NACC = NT == 128 ? 2 : 1;                  // accumulators (main / comp passes apart when they fit)
+  static constexpr int ACC_COLS = NACC * NT;
+  static constexpr int SFB_COLS = CH * 4 * (NT / 128);
+  static constexpr int SF_COLS = CH * 4 + SFB_COLS;               // per operand ring slot: A and B scale factors of a stage
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int NUM_BARS = 2 * WSTAGES + 2 * XSTAGES + 2 * ASTAGES + 4;
+  static constexpr size_t SMEM_BYTES =
+      1024 + (size_t)WSTAGES * W_BYTES + (size_t)XSTAGES * X_BYTES + (size_t)ASTAGES * ASTAGE_BYTES + NUM_BARS * 8 + 64;
+  // E2M1 x E2M1 -> FP32, UE4M3 scale factors, both operands K-major, M = 128, N = NT
+  static constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  static_assert(W_BYTES % 1024 == 0 && X_BYTES % 1024 == 0 && ASTAGE_BYTES % 1024 == 0, "swizzled tiles sit on 1024 bytes");
+  static_assert(ACC_COLS + ASTAGES * SF_COLS <= TMEM_COLS, "TMEM budget");
+  static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+};
 
 struct Args {
   __nv_bfloat16* y;
-  const uint8_t* sfb;        // activation scale factors: [token tile][stage][chunk] tiles of 512 bytes
+  const uint8_t* sfb;        // activation scale factors: [128-token tile][stage][chunk] tiles of 512 bytes
   float* slots;              // [grid][2][NT][128] FP32 partial tiles
   uint32_t* counters;        // one per output tile, zero between calls
   uint32_t* status;          // device status word
@@ -106,24 +116,41 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
 // writes made through the generic proxy become visible to the tensor core's (asynchronous proxy) reads
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Instruction descriptor: E2M1 x E2M1 -> FP32, UE4M3 scale factors, both operands K-major, M = 128, N = NT.
-constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 // Upper half of an operand's shared-memory descriptor: 1024-byte group stride, descriptor version, 128-byte swizzle.
 constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
 
+// Position of a role inside the CTA's stripe of work items, with the slot and parity of each ring.
+template <int XSTAGES>
+struct Cursor {
+  int tile, step;
+  int ws, wph, xs, xph, as, aph;
+  __device__ __forceinline__ void next(int steps_per_tile) {
+    if (++step == steps_per_tile) { step = 0; ++tile; }
+    if (++ws == WSTAGES) { ws = 0; wph ^= 1; }
+    if (++xs == XSTAGES) { xs = 0; xph ^= 1; }
+    if (++as == ASTAGES) { as = 0; aph ^= 1; }
+  }
+};
+
+template <int NT>
 __global__ void __launch_bounds__(THREADS, 1)
 razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Args a) {
+  using C = Cfg<NT>;
+  constexpr int XSTAGES = C::XSTAGES;
+  constexpr int X_WARP = 2 + NRW;                       // the activation producer
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* smem_a = smem + (size_t)STAGES * STAGE_BYTES;
+  uint8_t* smem_w = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* smem_x = smem_w + (size_t)WSTAGES * W_BYTES;
+  uint8_t* smem_a = smem_x + (size_t)XSTAGES * C::X_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_a + (size_t)ASTAGES * ASTAGE_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  uint32_t* bcast = tmem_slot + 2;
 
-  const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> remap, MMA
-  const uint32_t bar_empty = bar_full + 8 * STAGES;     // [STAGES]  MMA commit -> TMA
-  const uint32_t bar_afull = bar_empty + 8 * STAGES;    // [ASTAGES] remap -> MMA
+  const uint32_t bar_wfull = smem_u32(bars);            // [WSTAGES] TMA -> remap
+  const uint32_t bar_wempty = bar_wfull + 8 * WSTAGES;  // [WSTAGES] remap group (256 threads) -> TMA
+  const uint32_t bar_xfull = bar_wempty + 8 * WSTAGES;  // [XSTAGES] TMA -> MMA
+  const uint32_t bar_xempty = bar_xfull + 8 * XSTAGES;  // [XSTAGES] MMA commit -> TMA
+  const uint32_t bar_afull = bar_xempty + 8 * XSTAGES;  // [ASTAGES] remap -> MMA
   const uint32_t bar_aempty = bar_afull + 8 * ASTAGES;  // [ASTAGES] MMA commit -> remap
   const uint32_t bar_accfull = bar_aempty + 8 * ASTAGES;
   const uint32_t bar_accempty = bar_accfull + 8;
@@ -136,15 +163,19 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   const int it_end = (int)((a.total_items * (cta + 1)) / grid);
   const int n_items = it_end - it_begin;
   const int spt = a.steps_per_tile;
-  ItemCursor cur;
+  Cursor<XSTAGES> cur;
   cur.tile = it_begin / spt;
   cur.step = it_begin - cur.tile * spt;
-  cur.stage = cur.phase = cur.astage = cur.aphase = 0;
+  cur.ws = cur.wph = cur.xs = cur.xph = cur.as = cur.aph = 0;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; ++i) {
-      mbar_init(bar_full + 8 * i, 1);
-      mbar_init(bar_empty + 8 * i, 1);
+    for (int i = 0; i < WSTAGES; ++i) {
+      mbar_init(bar_wfull + 8 * i, 1);
+      mbar_init(bar_wempty + 8 * i, 256);
+    }
+    for (int i = 0; i < XSTAGES; ++i) {
+      mbar_init(bar_xfull + 8 * i, 1);
+      mbar_init(bar_xempty + 8 * i, 1);
     }
     for (int i = 0; i < ASTAGES; ++i) {
       mbar_init(bar_afull + 8 * i, 256);
@@ -158,45 +189,26 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     tmem_slot[3] = 0;                                   // a flag nobody sets (used by the drain waits)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // Producer state (thread 0 only).  The first ring of weight loads goes out before the rest of the prologue;
-  // the activation side (written by the preparation kernel) follows once that kernel has finished.
+  // Weight producer state (thread 0 only).  The first ring of weight loads goes out before the rest of the
+  // prologue: the packed weights depend on nothing that precedes this kernel in the stream.
   int issued = 0;
   int p_rt = cur.tile / a.token_tiles, p_tt = cur.tile - p_rt * a.token_tiles;
-  auto produce_x = [&](int stage, int step, int tt) {
-    const uint32_t st = smem_u32(smem) + (uint32_t)stage * STAGE_BYTES;
-    const uint32_t bar = bar_full + 8 * stage;
-    tma_load_2d(st + W_BYTES, &tmap_x, step * 128, tt * NT, bar);
-    bulk_copy_g2s(st + W_BYTES + X_BYTES, a.sfb + ((size_t)tt * spt + step) * SF_BYTES, SF_BYTES, bar);
-  };
-  auto produce = [&](bool with_x) {
-    const uint32_t st = smem_u32(smem) + (uint32_t)cur.stage * STAGE_BYTES;
-    const uint32_t bar = bar_full + 8 * cur.stage;
-    // the weight box always spans CH chunks (zero-filled past the end of K)
-    mbar_expect_tx(bar, (uint32_t)(W_BYTES + X_BYTES + SF_BYTES));
+  auto produce_w = [&]() {
+    const uint32_t st = smem_u32(smem_w) + (uint32_t)cur.ws * W_BYTES;
+    const uint32_t bar = bar_wfull + 8 * cur.ws;
+    mbar_expect_tx(bar, (uint32_t)W_BYTES);               // the box always spans CH chunks (zero-filled past the end of K)
     tma_load_3d(st, &tmap_w, 0, cur.step * CH, p_rt * TILE_STRIPS, bar);
-    if (with_x) produce_x(cur.stage, cur.step, p_tt);
     if (cur.step == spt - 1 && ++p_tt == a.token_tiles) { p_tt = 0; ++p_rt; }
-    cur.template next<STAGES, ASTAGES>(spt);
+    cur.next(spt);
   };
   if (threadIdx.x == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_w) : "memory");
     grid_dep_launch();
-    const ItemCursor first = cur;
-    const int first_tt = p_tt;
-    for (; issued < n_items && issued < STAGES; ++issued) produce(false);
-    grid_dep_wait();
-    ItemCursor c2 = first;
-    int tt2 = first_tt;
-    for (int i = 0; i < issued; ++i) {
-      produce_x(c2.stage, c2.step, tt2);
-      if (c2.step == spt - 1 && ++tt2 == a.token_tiles) tt2 = 0;
-      c2.template next<STAGES, ASTAGES>(spt);
-    }
+    for (; issued < n_items && issued < WSTAGES; ++issued) produce_w();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)TMEM_COLS)
+                 "r"((uint32_t)C::TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -204,7 +216,7 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_sf0 = tmem_base + ACC_COLS;
+  const uint32_t tmem_sf0 = tmem_base + C::ACC_COLS;
 
   auto fail = [&](uint32_t code) {
     *abort_flag = 1;
@@ -213,16 +225,40 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   };
 
   if (warp == 0) {
-    // ===================== TMA producer =====================
+    // ===================== weight producer =====================
     if (lane == 0) {
       for (; issued < n_items; ++issued) {
-        if (!mbar_wait(bar_empty + 8 * cur.stage, (uint32_t)cur.phase ^ 1u, abort_flag)) { fail(21); break; }
-        produce(true);
+        if (!mbar_wait(bar_wempty + 8 * cur.ws, (uint32_t)cur.wph ^ 1u, abort_flag)) { fail(21); break; }
+        produce_w();
       }
       // copies still in flight must land before this CTA's shared memory is released
-      const int pending = issued < STAGES ? issued : STAGES;
+      const int pending = issued < WSTAGES ? issued : WSTAGES;
       for (int f = issued - pending; f < issued; ++f)
-        mbar_wait(bar_full + 8 * (f % STAGES), (uint32_t)((f / STAGES) & 1), tmem_slot + 3);
+        mbar_wait(bar_wfull + 8 * (f % WSTAGES), (uint32_t)((f / WSTAGES) & 1), tmem_slot + 3);
+    }
+  } else if (warp == X_WARP) {
+    // ===================== activation producer (codes and scale factors written by the preparation kernel) =====================
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+      grid_dep_wait();
+      int tt = cur.tile % a.token_tiles;
+      int done = 0;
+      for (; done < n_items; ++done) {
+        if (done >= XSTAGES && !mbar_wait(bar_xempty + 8 * cur.xs, (uint32_t)cur.xph ^ 1u, abort_flag)) { fail(22); break; }
+        const uint32_t st = smem_u32(smem_x) + (uint32_t)cur.xs * C::X_BYTES;
+        const uint32_t bar = bar_xfull + 8 * cur.xs;
+        mbar_expect_tx(bar, (uint32_t)C::X_BYTES);
+        tma_load_2d(st, &tmap_x, cur.step * 128, tt * NT, bar);
+#pragma unroll
+        for (int h = 0; h < NT / 128; ++h)
+          bulk_copy_g2s(st + C::X_CODE_BYTES + h * SF_BYTES,
+                        a.sfb + ((size_t)(tt * (NT / 128) + h) * spt + cur.step) * SF_BYTES, SF_BYTES, bar);
+        if (cur.step == spt - 1 && ++tt == a.token_tiles) tt = 0;
+        cur.next(spt);
+      }
+      const int pending = done < XSTAGES ? done : XSTAGES;
+      for (int f = done - pending; f < done; ++f)
+        mbar_wait(bar_xfull + 8 * (f % XSTAGES), (uint32_t)((f / XSTAGES) & 1), tmem_slot + 3);
     }
   } else if (warp == 1) {
     // ===================== MMA issuer (whole warp walks the items, one elected lane issues) =====================
@@ -236,46 +272,48 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       const bool seg_first = (i == 0) || cur.step == 0;
       const bool seg_last = (i + 1 == n_items) || cur.step == spt - 1;
       const int nch = min(CH, a.g.k_chunks - cur.step * CH);
-      // the group that filled this operand slot waited for the shared-memory stage before it read it, so its
-      // arrival also covers the stage's activation codes and scale factors
-      if (!wait_warp(bar_afull + 8 * cur.astage, (uint32_t)cur.aphase, 23)) break;
+      if (!wait_warp(bar_afull + 8 * cur.as, (uint32_t)cur.aph, 23)) break;
+      if (!wait_warp(bar_xfull + 8 * cur.xs, (uint32_t)cur.xph, 30)) break;
       if (seg_first && !wait_warp(bar_accempty, (seg & 1u) ^ 1u, 24)) break;
       tc_fence_after();
-      const uint32_t xs = smem_u32(smem) + (uint32_t)cur.stage * STAGE_BYTES + W_BYTES;
-      const uint32_t sfb_s = xs + X_BYTES;
-      const uint32_t am = smem_u32(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES;
+      const uint32_t xs = smem_u32(smem_x) + (uint32_t)cur.xs * C::X_BYTES;
+      const uint32_t sfb_s = xs + C::X_CODE_BYTES;
+      const uint32_t am = smem_u32(smem_a) + (uint32_t)cur.as * ASTAGE_BYTES;
       const uint32_t ac = am + A_TILE_BYTES;
       const uint32_t sfa_s = am + 2 * A_TILE_BYTES;
-      const uint32_t sf_t = tmem_sf0 + cur.astage * SF_COLS;
+      const uint32_t sf_t = tmem_sf0 + cur.as * C::SF_COLS;
       if (elect_one()) {
         // the stage's scale factors first, then its MMAs back to back
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           if (c < nch) {
             copy_sf_to_tmem(sf_t + c * 4, sfa_s + c * SF_TILE_BYTES);
-            copy_sf_to_tmem(sf_t + CH * 4 + c * 4, sfb_s + c * SF_TILE_BYTES);
+#pragma unroll
+            for (int h = 0; h < NT / 128; ++h)
+              copy_sf_to_tmem(sf_t + CH * 4 + c * 4 * (NT / 128) + h * 4, sfb_s + h * SF_BYTES + c * SF_TILE_BYTES);
           }
         }
-        // Main and comp passes add into accumulators of their own (summed in the epilogue): MMAs on one
-        // accumulator execute one after the other, and consecutive MMAs then never share one.
+        // With two accumulators the main and comp passes add into one each (summed in the epilogue), so that
+        // consecutive MMAs never share an accumulator.
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           if (c < nch) {
-            const uint32_t sfa_t = sf_t + c * 4, sfb_t = sf_t + CH * 4 + c * 4;
+            const uint32_t sfa_t = sf_t + c * 4, sfb_t = sf_t + CH * 4 + c * 4 * (NT / 128);
             // 64 codes further along k: +32 bytes inside the 128-byte rows
             const uint32_t b_lo = ((xs + c * 32) >> 4) | (1u << 16);
-            const uint32_t acc = (seg_first && c == 0) ? 0u : 1u;
-            mma_fp4(tmem_base, ((am + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t, acc);
-            mma_fp4(tmem_base + NT, ((ac + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, IDESC, sfa_t, sfb_t, acc);
+            const uint32_t first = (seg_first && c == 0) ? 0u : 1u;
+            mma_fp4(tmem_base, ((am + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, C::IDESC, sfa_t, sfb_t, first);
+            mma_fp4(tmem_base + (C::NACC - 1) * NT, ((ac + c * 32) >> 4) | (1u << 16), b_lo, DESC_HI, C::IDESC, sfa_t, sfb_t,
+                    C::NACC == 2 ? first : 1u);
           }
         }
-        tc_commit(bar_empty + 8 * cur.stage);
-        tc_commit(bar_aempty + 8 * cur.astage);
+        tc_commit(bar_xempty + 8 * cur.xs);
+        tc_commit(bar_aempty + 8 * cur.as);
         if (seg_last) tc_commit(bar_accfull);
       }
       __syncwarp();
       if (seg_last) ++seg;
-      cur.template next<STAGES, ASTAGES>(spt);
+      cur.next(spt);
     }
     // the MMAs issued so far read shared memory and TMEM until they complete: wait for them (bounded, not
     // watching the abort flag) before the CTA may release either
@@ -292,7 +330,7 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int group = (warp - 2) >> 3;
     const int half = ((warp - 2) >> 2) & 1;
     constexpr int GROUPS = NRW / 8;
-    static_assert(GROUPS == ASTAGES && STAGES >= ASTAGES, "an operand slot per group; see the wait order below");
+    static_assert(GROUPS == ASTAGES && WSTAGES % GROUPS == 0, "an operand slot per group; a weight stage always serves the same group");
     constexpr int EPI_SETS = NRW / 4;                     // sets of four warps (all lane quarters) share the columns
     const int col_lo = 16 * ((((warp - 2) >> 2) * (NT / 16)) / EPI_SETS);
     const int col_hi = 16 * (((((warp - 2) >> 2) + 1) * (NT / 16)) / EPI_SETS);
@@ -322,20 +360,19 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t sw7 = (uint32_t)row & 7u;              // 128-byte swizzle: 16-byte unit u of row r sits at u ^ (r % 8)
     const uint32_t sf_word = (uint32_t)((row & 31) * 4 + (row >> 5)) * 4;
     int turn = 0;                                        // item i is remapped by group i % GROUPS
-    for (int i = 0; i < n_items; ++i, cur.template next<STAGES, ASTAGES>(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
+    for (int i = 0; i < n_items; ++i, cur.next(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
       const int tile = cur.tile, step = cur.step;
       const bool seg_last = (i + 1 == n_items) || step == spt - 1;
       const int nch = min(CH, a.g.k_chunks - step * CH);
       if (turn == group) {
-        // The operand slot is this group's own, and its release by the MMA warp (which takes the items in
-        // order) means that every item up to i - ASTAGES was issued, hence remapped, hence landed: the stage's
-        // previous fill (item i - STAGES, STAGES >= ASTAGES) among them, so the parity wait on it is sound.
-        if (!wait_all(bar_aempty + 8 * cur.astage, (uint32_t)cur.aphase ^ 1u, 26)) break;
-        if (!wait_all(bar_full + 8 * cur.stage, (uint32_t)cur.phase, 25)) break;
-        const uint32_t st = smem_addr(smem) + (uint32_t)cur.stage * STAGE_BYTES + strip_off;
-        const uint32_t am = smem_addr(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES + row_off;
+        // The operand slot and (WSTAGES being a multiple of GROUPS) the weight stage always serve this group, so
+        // the group sees every phase of both barriers and its parity waits are sound.
+        if (!wait_all(bar_aempty + 8 * cur.as, (uint32_t)cur.aph ^ 1u, 26)) break;
+        if (!wait_all(bar_wfull + 8 * cur.ws, (uint32_t)cur.wph, 25)) break;
+        const uint32_t st = smem_addr(smem_w) + (uint32_t)cur.ws * W_BYTES + strip_off;
+        const uint32_t am = smem_addr(smem_a) + (uint32_t)cur.as * ASTAGE_BYTES + row_off;
         const uint32_t ac = am + A_TILE_BYTES;
-        const uint32_t sfa = smem_addr(smem_a) + (uint32_t)cur.astage * ASTAGE_BYTES + 2 * A_TILE_BYTES + sf_word;
+        const uint32_t sfa = smem_addr(smem_a) + (uint32_t)cur.as * ASTAGE_BYTES + 2 * A_TILE_BYTES + sf_word;
 #pragma unroll
         for (int cc = 0; cc < CH / 2; ++cc) {
           const int c = half * (CH / 2) + cc;
@@ -370,8 +407,9 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             sts32(sfa + c * SF_TILE_BYTES, sw & 0x3F3F3F3Fu);
           }
         }
+        mbar_arrive(bar_wempty + 8 * cur.ws);               // the packed bytes are in registers or written out
         fence_async_smem();
-        mbar_arrive(bar_afull + 8 * cur.astage);
+        mbar_arrive(bar_afull + 8 * cur.as);
       }
 
       if (!seg_last) continue;
@@ -413,12 +451,17 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       float* my_slot = a.slots + (size_t)cta * 2 * (size_t)(NT * TILE_ROWS);   // a non-owner's part is its stripe's first segment
 #pragma unroll 1
       for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
-        uint32_t v[16], v1[16];
+        uint32_t v[16];
         tc_ld16(tmem_base + lane_off + c0, v);
-        tc_ld16(tmem_base + lane_off + NT + c0, v1);
-        tc_wait_ld();
+        if (C::NACC == 2) {
+          uint32_t v1[16];
+          tc_ld16(tmem_base + lane_off + NT + c0, v1);
+          tc_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v1[j]));
+          for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v1[j]));
+        } else {
+          tc_wait_ld();
+        }
         if (complete || owner) {
           if (owner) {
             const int m_valid = a.M - (m0 + c0);                       // tokens of this column group that exist
@@ -470,24 +513,24 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS)
                  : "memory");
   }
 }
 
 // Activation operand for the kernel above.  codes_out: [M][KP / 8] 32-bit words (KP = K rounded up to whole
 // stages, zero beyond K), each word's nibbles in the packed form's order (nibbles p and p + 4 = elements 2p and
-// 2p + 1).  sfb: [token tile][stage][chunk] tiles of 128 words; word 4 * (t % 32) + t / 32 of a tile holds the
+// 2p + 1).  sfb: [128-token tile][stage][chunk] tiles of 128 words; word 4 * (t % 32) + t / 32 of a tile holds the
 // four 7-bit scale bytes of token t of the tile for the chunk's four blocks (zero for tokens beyond M and
 // blocks beyond K).
 __global__ void fp4_act_prep_kernel(const uint32_t* __restrict__ codes, const uint8_t* __restrict__ scales, int M, int K,
-                                    int KP, int token_tiles, int spt, uint32_t* __restrict__ codes_out,
+                                    int KP, int tiles128, int spt, uint32_t* __restrict__ codes_out,
                                     uint32_t* __restrict__ sfb) {
   grid_dep_launch();
   grid_dep_wait();
   const long long row_words = KP / 8, in_words = K / 8;
   const long long n_code = (long long)M * row_words;
-  const long long n_sf = (long long)token_tiles * spt * CH * 128;
+  const long long n_sf = (long long)tiles128 * spt * CH * 128;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_code + n_sf;
        i += (long long)gridDim.x * blockDim.x) {
     if (i < n_code) {
@@ -504,7 +547,7 @@ __global__ void fp4_act_prep_kernel(const uint32_t* __restrict__ codes, const ui
       const int c = (int)(tile % CH);
       const int step = (int)((tile / CH) % spt);
       const int tt = (int)(tile / ((long long)CH * spt));
-      const int token = tt * NT + (wi >> 2) + 32 * (wi & 3);
+      const int token = tt * 128 + (wi >> 2) + 32 * (wi & 3);
       const int kb0 = (step * CH + c) * 4;
       uint32_t v = 0;
       if (token < M) {
@@ -518,7 +561,7 @@ __global__ void fp4_act_prep_kernel(const uint32_t* __restrict__ codes, const ui
 }
 
 struct Plan {
-  int token_tiles, steps_per_tile, grid, KP;
+  int NT, token_tiles, tiles128, steps_per_tile, grid, KP;
   long long tiles, total_items;
   size_t counters_bytes, slots_bytes, codes_bytes, sfb_bytes;
 };
@@ -526,7 +569,9 @@ struct Plan {
 static Plan make_plan(const razer_desc* d, int M) {
   Plan p;
   const Geometry g = make_geometry(d->N, d->K);
-  p.token_tiles = (M + NT - 1) / NT;
+  p.NT = M > 128 ? 256 : 128;
+  p.token_tiles = (M + p.NT - 1) / p.NT;
+  p.tiles128 = p.token_tiles * (p.NT / 128);
   p.steps_per_tile = (g.k_chunks + CH - 1) / CH;
   p.KP = p.steps_per_tile * CH * CHUNK_K;
   p.tiles = (long long)g.row_tiles * p.token_tiles;
@@ -534,9 +579,9 @@ static Plan make_plan(const razer_desc* d, int M) {
   const int sms = sm_count();
   p.grid = (int)(p.total_items < sms ? p.total_items : sms);
   p.counters_bytes = align256((size_t)p.tiles * sizeof(uint32_t));
-  p.slots_bytes = (size_t)(p.grid > 148 ? p.grid : 148) * 2 * NT * TILE_ROWS * sizeof(float);
+  p.slots_bytes = (size_t)(p.grid > 148 ? p.grid : 148) * 2 * p.NT * TILE_ROWS * sizeof(float);
   p.codes_bytes = align256((size_t)M * p.KP / 2);
-  p.sfb_bytes = (size_t)p.token_tiles * p.steps_per_tile * SF_BYTES;
+  p.sfb_bytes = (size_t)p.tiles128 * p.steps_per_tile * SF_BYTES;
   return p;
 }
 
@@ -626,7 +671,7 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
     // padded activation codes as bytes: [M][KP / 2]; box = 128 bytes (one stage of k) x NT tokens
     const cuuint64_t dims[2] = {(cuuint64_t)(p.KP / 2), (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)(p.KP / 2)};
-    const cuuint32_t box[2] = {128, (cuuint32_t)NT};
+    const cuuint32_t box[2] = {128, (cuuint32_t)p.NT};
     const CUresult r = enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, codes_pad, dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -646,7 +691,7 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   {
-    const long long work = (long long)M * (p.KP / 8) + (long long)p.token_tiles * p.steps_per_tile * CH * 128;
+    const long long work = (long long)M * (p.KP / 8) + (long long)p.tiles128 * p.steps_per_tile * CH * 128;
     long long blocks = (work + 255) / 256;
     if (blocks > 148 * 8) blocks = 148 * 8;
     cudaLaunchConfig_t cfg = {};
@@ -656,24 +701,36 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, fp4_act_prep_kernel, (const uint32_t*)act_codes, act_scales, M, d->K, p.KP,
-                                             p.token_tiles, p.steps_per_tile, (uint32_t*)codes_pad, (uint32_t*)sfb);
+                                             p.tiles128, p.steps_per_tile, (uint32_t*)codes_pad, (uint32_t*)sfb);
     count_launches(1);
     RAZER_TRY(check_cuda(e, "fp4_act_prep_kernel launch"));
-  }
-  static bool attr_set = false;
-  if (!attr_set) {
-    RAZER_TRY(check_cuda(cudaFuncSetAttribute(razer_fp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES),
-                         "cudaFuncSetAttribute(max dynamic shared memory)"));
-    attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)p.grid);
   cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, razer_fp4_kernel, tmap_x, tmap_w, a);
+  cudaError_t e;
+  if (p.NT == 128) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      RAZER_TRY(check_cuda(cudaFuncSetAttribute(razer_fp4_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)Cfg<128>::SMEM_BYTES), "cudaFuncSetAttribute(max dynamic shared memory)"));
+      attr_set = true;
+    }
+    cfg.dynamicSmemBytes = Cfg<128>::SMEM_BYTES;
+    e = cudaLaunchKernelEx(&cfg, razer_fp4_kernel<128>, tmap_x, tmap_w, a);
+  } else {
+    static bool attr_set = false;
+    if (!attr_set) {
+      RAZER_TRY(check_cuda(cudaFuncSetAttribute(razer_fp4_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)Cfg<256>::SMEM_BYTES), "cudaFuncSetAttribute(max dynamic shared memory)"));
+      attr_set = true;
+    }
+    cfg.dynamicSmemBytes = Cfg<256>::SMEM_BYTES;
+    e = cudaLaunchKernelEx(&cfg, razer_fp4_kernel<256>, tmap_x, tmap_w, a);
+  }
   count_launches(1);
   return check_cuda(e, "razer_fp4_kernel launch");
 }
