@@ -201,13 +201,22 @@ def run_shape(args):
     desc, sets, _ = make_sets(b, torch, inputs, N, K, 2, 7)
     x = inputs.activations(M, K, 3).cuda()
     y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
-    fn, op = (b.razer_gemv, b.OP_GEMV) if M <= 64 else (b.razer_gemm, b.OP_GEMM)
-    ws = b.alloc_workspace(desc, M, op, "cuda")
+    if args.op == "auto":
+        fn, op = (b.razer_gemv, b.OP_GEMV) if M <= 64 else (b.razer_gemm, b.OP_GEMM)
+        name = "razer_gemv" if M <= 64 else "razer_gemm"
+        ws = b.alloc_workspace(desc, M, op, "cuda")
+        call = lambda i: fn(desc, sets[i % 2], x, y, ws)
+    else:
+        native = args.op == "w4a4-fp4"
+        name = "razer_gemm_w4a4 (two-pass block-scaled FP4)" if native else "razer_gemm_w4a4"
+        ws = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+        ac, as_, ats = b.razer_quant_act(x, sv_mag=0.0 if native else 5.0)
+        call = lambda i: b.razer_gemm_w4a4(desc, sets[i % 2], ac, as_, ats, y=y, workspace=ws, use_native_fp4=native)
     for i in range(args.warmup):
-        fn(desc, sets[i % 2], x, y, ws)
-    ms = time_cuda(lambda i: fn(desc, sets[i % 2], x, y, ws), args.steps, torch)
+        call(i)
+    ms = time_cuda(call, args.steps, torch)
     b.razer_workspace_status(ws)
-    print(json.dumps({"shape": [M, N, K], "op": "razer_gemv" if M <= 64 else "razer_gemm", "us_per_launch_stream": ms * 1e3,
+    print(json.dumps({"shape": [M, N, K], "op": name, "us_per_launch_stream": ms * 1e3,
                       "launches": args.warmup + args.steps, "algorithmic_bytes": algo_bytes(M, N, K),
                       "flops": 2.0 * M * N * K}))
 
@@ -224,6 +233,7 @@ def main():
     ap.add_argument("--window-ms", type=float, default=200.0, help="length of a timed window (0: one graph replay)")
     ap.add_argument("--shape", default="", help="MxNxK: time that one matmul alone (a small, single-kernel run for "
                                                 "profiler captures); prints its own short JSON line, not the bench line")
+    ap.add_argument("--op", default="auto", help="with --shape: auto (razer_gemv / razer_gemm by M), w4a4 or w4a4-fp4")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

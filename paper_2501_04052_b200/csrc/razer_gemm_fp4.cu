@@ -9,11 +9,13 @@
 // is the hardware's UE4M3 scale factor as it stands.  The two passes are two MMAs per 64-column chunk into
 // the same TMEM accumulator; neither matrix exists in global memory.
 //
-// Mapping: the weight tile is the MMA's A operand (128 rows), the token tile its B operand (128 tokens),
-// both K-major FP4 in shared memory with the 128-byte swizzle (one row = 256 codes = one stage of four
-// chunks).  Warp 0 = TMA producer (packed weights, activation codes, activation scale factors), warp 1 =
-// TMEM owner and MMA issuer, warps 2..17 = remap (thread = weight row and half of a stage's chunks; two groups of eight warps take
-// the stages in turn) and epilogue.  A remap thread reads its row's packed blocks, finds the special-value
+// Mapping: the weight tile is the MMA's A operand (128 rows), the token tile its B operand (128 tokens, or 256
+// when there are more than 128), both K-major FP4 in shared memory with the 128-byte swizzle (one row = 256
+// codes = one stage of four chunks).  Warp 0 = weight producer (TMA box of packed bytes into a ring of its own,
+// released by the remap warps as soon as they have read it), warp 1 = TMEM owner and MMA issuer, warps 2..17 =
+// remap (thread = weight row and half of a stage's chunks; two groups of eight warps take the stages in turn)
+// and epilogue, warp 18 = activation producer (codes by TMA, scale-factor tiles by bulk copy, into a ring
+// released by the MMAs' completion).  A remap thread reads its row's packed blocks, finds the special-value
 // nibbles (the only nibbles that are 0x0 in the packed form), builds the two code words with two integer
 // multiply-adds, applies the block's stored-negated flag to the sign bits, and writes both rows plus the row's
 // four scale bytes (scale-factor layout: 32 x 16-byte rows, row r % 32, word r / 32).  The MMA warp copies
@@ -528,18 +530,31 @@ __global__ void fp4_act_prep_kernel(const uint32_t* __restrict__ codes, const ui
                                     uint32_t* __restrict__ sfb) {
   grid_dep_launch();
   grid_dep_wait();
-  const long long row_words = KP / 8, in_words = K / 8;
-  const long long n_code = (long long)M * row_words;
+  const long long row_quads = KP / 32, in_words = K / 8;               // a quad = four 32-bit words = 32 codes
+  const long long n_code = (long long)M * row_quads;
   const long long n_sf = (long long)tiles128 * spt * CH * 128;
+  const bool vec = (K % 32) == 0 && (reinterpret_cast<uintptr_t>(codes) % 16) == 0;   // rows of the input start on 16 bytes
+  auto shuffle = [](uint32_t w) -> uint32_t {                          // element j of the word: nibble j -> nibble j / 2 + 4 (j % 2)
+    uint32_t o = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) o |= ((w >> (4 * j)) & 0xFu) << (4 * ((j >> 1) + 4 * (j & 1)));
+    return o;
+  };
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_code + n_sf;
        i += (long long)gridDim.x * blockDim.x) {
     if (i < n_code) {
-      const long long m = i / row_words, wi = i - m * row_words;
-      const uint32_t w = wi < in_words ? codes[m * in_words + wi] : 0u;
-      uint32_t o = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) o |= ((w >> (4 * j)) & 0xFu) << (4 * ((j >> 1) + 4 * (j & 1)));
-      codes_out[i] = o;
+      const long long m = i / row_quads, q = i - m * row_quads;
+      uint4 w = make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t* src = codes + m * in_words + 4 * q;
+      if (vec && 4 * q + 3 < in_words) {
+        w = *reinterpret_cast<const uint4*>(src);
+      } else {
+        if (4 * q + 0 < in_words) w.x = src[0];
+        if (4 * q + 1 < in_words) w.y = src[1];
+        if (4 * q + 2 < in_words) w.z = src[2];
+        if (4 * q + 3 < in_words) w.w = src[3];
+      }
+      reinterpret_cast<uint4*>(codes_out)[i] = make_uint4(shuffle(w.x), shuffle(w.y), shuffle(w.z), shuffle(w.w));
     } else {
       const long long s = i - n_code;
       const int wi = (int)(s & 127);
@@ -570,6 +585,10 @@ static Plan make_plan(const razer_desc* d, int M) {
   Plan p;
   const Geometry g = make_geometry(d->N, d->K);
   p.NT = M > 128 ? 256 : 128;
+  if (const char* e = getenv("RAZER_FP4_NT")) {                       // tuning and test aid: force the token tile
+    const int v = atoi(e);
+    if (v == 128 || v == 256) p.NT = v;
+  }
   p.token_tiles = (M + p.NT - 1) / p.NT;
   p.tiles128 = p.token_tiles * (p.NT / 128);
   p.steps_per_tile = (g.k_chunks + CH - 1) / CH;
@@ -691,7 +710,7 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   {
-    const long long work = (long long)M * (p.KP / 8) + (long long)p.tiles128 * p.steps_per_tile * CH * 128;
+    const long long work = (long long)M * (p.KP / 32) + (long long)p.tiles128 * p.steps_per_tile * CH * 128;
     long long blocks = (work + 255) / 256;
     if (blocks > 148 * 8) blocks = 148 * 8;
     cudaLaunchConfig_t cfg = {};

@@ -381,6 +381,20 @@ def test_w4a4_native_fp4_two_pass(b, M, N, K, sv_mag, remap_code):
     _w4a4_native_check(b, desc, packed, wc, ws, wd, ac, as_, ats, sv_mag=sv_mag, remap_code=remap_code)
 
 
+@pytest.mark.parametrize("nt,M", [(128, 300), (256, 40), (256, 300)])
+def test_w4a4_native_fp4_forced_token_tile(b, monkeypatch, nt, M):
+    """Both token-tile widths of the FP4 kernel at token counts the host would give to the other one."""
+    monkeypatch.setenv("RAZER_FP4_NT", str(nt))
+    N, K = 390, 2320                                                   # ragged row tile, 9.06 stages
+    w = inputs.student_t_weights(N, K, 310 + nt, outlier_frac=0.001).numpy()
+    wc, ws, wd = ro.quantize_weight(w)
+    desc = b.make_desc(N, K, float(wd))
+    packed = b.razer_pack_layout(desc, torch.from_numpy(wc).cuda(), torch.from_numpy(ws).cuda())
+    x = inputs.activations(M, K, 311, outlier_channel_frac=0.01)
+    ac, as_, ats = b.razer_quant_act(x.cuda(), sv_mag=0.0)
+    _w4a4_native_check(b, desc, packed, wc, ws, wd, ac, as_, ats)
+
+
 def test_w4a4_native_fp4_decodes_bit_exactly(b):
     """One-hot NVFP4 activations (code 1.0, block scale 1.0) through the two-pass path: y[m, n] is the tensor
     scale times one decoded weight, exact whatever the accumulation order, so main + comp is checked bit for bit."""
