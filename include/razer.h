@@ -26,6 +26,14 @@
  *   passed as void* (NULL = the default stream).  bf16 tensors are raw 16-bit patterns.
  *   Every function returns RAZER_OK (0) or a negative RAZER_ERR_* code, never throws;
  *   razer_last_error() returns a description of the calling thread's last failure.
+ *   Stream ordering: the matmul kernels are launched with programmatic dependent launch
+ *   (RAZER_PDL=0 in the environment turns it off).  They read the PACKED WEIGHTS before the
+ *   kernel directly ahead of them on the stream is known to have finished, and everything
+ *   else (activations, outputs, workspace, scale scalars) after it.  Guaranteed: weights
+ *   written by razer_pack_layout, by a copy (cudaMemcpyAsync) or by anything that is not the
+ *   immediately preceding kernel of the stream are seen.  Not guaranteed: weights written by
+ *   a caller's own kernel launched directly ahead of the matmul; put any other operation
+ *   between the two (razer_pack_layout does so itself).
  */
 #ifndef RAZER_H_
 #define RAZER_H_

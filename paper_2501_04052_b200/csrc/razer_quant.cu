@@ -249,13 +249,18 @@ __global__ void quant_weight_kernel(const float4* __restrict__ w, long long n_bl
         const float xv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
+          // the four standard candidates share the scale of Eq. 2, hence the scaled value and its FP4 rounding
+          float xs = 0.0f, r = 0.0f, d_r = 0.0f;
 #pragma unroll
           for (int c = 0; c < NC; ++c) {
             if (c >= 4 && !ok[c]) continue;
-            const float xs = __fdiv_rn(xv[j], cd[c]);                  // the scaled block of Eq. 6
-            const uint32_t idx = round_to_fp4_idx(fabsf(xs));
-            const float r = (__float_as_uint(xs) >> 31) ? -fp4_mag(idx) : fp4_mag(idx);
-            const bool tk = fabsf(__fsub_rn(xs, cv[c])) < fabsf(__fsub_rn(xs, r));   // strictly closer only
+            if (c == 0 || c >= 4) {
+              xs = __fdiv_rn(xv[j], cd[c]);                            // the scaled block of Eq. 6
+              const uint32_t idx = round_to_fp4_idx(fabsf(xs));
+              r = (__float_as_uint(xs) >> 31) ? -fp4_mag(idx) : fp4_mag(idx);
+              d_r = fabsf(__fsub_rn(xs, r));
+            }
+            const bool tk = fabsf(__fsub_rn(xs, cv[c])) < d_r;         // strictly closer only
             const float d = __fsub_rn(tk ? cv[c] : r, xs);
             err[c] = __fadd_rn(err[c], __fmul_rn(d, d));               // ascending element order, no fusion
           }

@@ -514,6 +514,38 @@ def test_workspace_too_small_is_an_error(b):
         assert e.value.code == b.ERR_WORKSPACE
 
 
+def test_weights_written_just_ahead_of_the_matmul_are_seen(b):
+    """Stream-ordering contract of the header: the matmul kernels start reading the packed weights before the kernel
+    directly ahead of them is known to have finished (programmatic dependent launch).  What is guaranteed: weights
+    written by razer_pack_layout or by a device-to-device copy queued directly ahead of the matmul are the ones read.
+    Two different tensors go alternately into ONE packed buffer, each time followed at once by the GEMV."""
+    N, K = 4096, 4096
+    desc = b.make_desc(N, K, 0.002)
+    sets, want = [], []
+    x = inputs.activations(1, K, 7).cuda()
+    ws = b.alloc_workspace(desc, 1, b.OP_GEMV, "cuda")
+    for s in range(2):
+        c, sc = inputs.random_codes(N, K, seed=400 + s)
+        sets.append((c.cuda(), sc.cuda()))
+        p = b.razer_pack_layout(desc, *sets[-1])
+        want.append(b.razer_gemv(desc, p, x, workspace=ws).clone())
+    assert not torch.equal(want[0], want[1])
+    packed = torch.empty_like(p)
+    y = torch.empty_like(want[0])
+    keep = [b.razer_pack_layout(desc, *sets[s]) for s in range(2)]
+    bad = 0
+    for i in range(300):
+        s = i & 1
+        if i % 3 == 0:
+            packed.copy_(keep[s])                                       # device-to-device copy
+        else:
+            b.razer_pack_layout(desc, sets[s][0], sets[s][1], packed)   # the library's own writer
+        b.razer_gemv(desc, packed, x, y, ws)
+        bad += int(not torch.equal(y, want[s]))
+    b.razer_workspace_status(ws)
+    assert bad == 0, f"{bad} of 300 launches read stale weights"
+
+
 # ------------------------------------------------------------------ alternative kernels (chosen by environment)
 
 _ALT_KERNEL_CHECK = r"""
