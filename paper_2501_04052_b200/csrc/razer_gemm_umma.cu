@@ -109,7 +109,6 @@ razer_umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(        // 16-byte aligned: the tables behind it are read as uint4
       (reinterpret_cast<uintptr_t>(bars + Cfg::NUM_BARS) + 15) & ~(uintptr_t)15);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  uint32_t* bcast = tmem_slot + 2;                      // epilogue broadcast word
   uint8_t* tables = reinterpret_cast<uint8_t*>(tmem_slot + 16);   // decode tables (razer_decode.cuh)
 
   const uint32_t bar_full = smem_u32(bars);             // [STAGES]  TMA -> dequant, MMA
