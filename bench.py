@@ -206,6 +206,11 @@ def run_shape(args):
         name = "razer_gemv" if M <= 64 else "razer_gemm"
         ws = b.alloc_workspace(desc, M, op, "cuda")
         call = lambda i: fn(desc, sets[i % 2], x, y, ws)
+    elif args.op == "w4a4-fp4-prepared":
+        name = "razer_gemm_w4a4_fp4 (two-pass block-scaled FP4, prepared operand)"
+        ws = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+        act4, ats4 = b.razer_quant_act_fp4(x)
+        call = lambda i: b.razer_gemm_w4a4_fp4(desc, sets[i % 2], act4, ats4, M, y=y, workspace=ws)
     else:
         native = args.op == "w4a4-fp4"
         name = "razer_gemm_w4a4 (two-pass block-scaled FP4)" if native else "razer_gemm_w4a4"
@@ -233,7 +238,8 @@ def main():
     ap.add_argument("--window-ms", type=float, default=200.0, help="length of a timed window (0: one graph replay)")
     ap.add_argument("--shape", default="", help="MxNxK: time that one matmul alone (a small, single-kernel run for "
                                                 "profiler captures); prints its own short JSON line, not the bench line")
-    ap.add_argument("--op", default="auto", help="with --shape: auto (razer_gemv / razer_gemm by M), w4a4 or w4a4-fp4")
+    ap.add_argument("--op", default="auto", help="with --shape: auto (razer_gemv / razer_gemm by M), w4a4, w4a4-fp4 "
+                                                 "(interchange-format activations) or w4a4-fp4-prepared")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -432,6 +438,20 @@ def main():
         extras.append({"config": 5, "op": "razer_gemm_w4a4 (two-pass block-scaled FP4)", "M": M, "N": N, "K": K,
                        "us": t4 * 1e3, "TFLOPs_effective": tf4, "frac_fp4_two_pass": 2.0 * tf4 / (4.0 * pk["bf16"]),
                        "GBps": algo_bytes(M, N, K) / (t4 * 1e-3) / 1e9, "frac_hbm": algo_bytes(M, N, K) / (t4 * 1e-3) / 1e9 / pk["hbm"]})
+        # the same with the quantizer writing the tensor core's operand layout itself (no re-layout kernel)
+        act4, ats4 = b.razer_quant_act_fp4(x)
+        tq4 = graph_time(lambda i: b.razer_quant_act_fp4(x, act_fp4=act4), 8)
+        f5 = lambda i: b.razer_gemm_w4a4_fp4(desc, sets[i % 4], act4, ats4, M, y=y, workspace=ws4)
+        for i in range(3):
+            f5(i)
+        t5 = graph_time(f5, 8)
+        tf5 = 2.0 * M * N * K / (t5 * 1e-3) / 1e12
+        extras.append({"config": 5, "op": "razer_quant_act_fp4", "M": M, "K": K, "us": tq4 * 1e3,
+                       "GBps": (M * K * 2 + M * K * 0.5625) / (tq4 * 1e-3) / 1e9})
+        extras.append({"config": 5, "op": "razer_gemm_w4a4_fp4 (two-pass block-scaled FP4, prepared operand)", "M": M, "N": N,
+                       "K": K, "us": t5 * 1e3, "TFLOPs_effective": tf5, "frac_fp4_two_pass": 2.0 * tf5 / (4.0 * pk["bf16"]),
+                       "frac_bf16_effective": tf5 / pk["bf16"], "GBps": algo_bytes(M, N, K) / (t5 * 1e-3) / 1e9,
+                       "frac_hbm": algo_bytes(M, N, K) / (t5 * 1e-3) / 1e9 / pk["hbm"]})
         # GPU weight quantizer (offline step; FP32 in, interchange format out), 4096 x 4096
         wq = inputs.student_t_weights(4096, 4096, 5000, outlier_frac=0.001).cuda()
         b.razer_quant_weight(wq)

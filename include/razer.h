@@ -234,6 +234,24 @@ int razer_gemm_w4a4(const razer_desc* d, const void* packed_w_dev, const uint8_t
                     int M, void* y_dev, void* workspace_dev, size_t workspace_bytes,
                     int use_native_fp4, void* stream);
 
+/* The same two-pass matmul with the activation operand produced directly in the layout the tensor core reads,
+ * the way App. D.3 generates B_main and B_comp "directly in the packed sub-byte layout" its GEMM consumes: no
+ * re-layout kernel between quantizer and matmul.
+ * razer_fp4_act_bytes: size of that operand for M x K activations (256-byte aligned buffer, caller-owned).
+ * razer_quant_act_fp4: plain NVFP4 quantization (Eq. 1-3, the arithmetic of razer_quant_act with sv_mag = 0; same
+ * tensor_scale_in_dev / amax_scratch_dev contract, one launch) writing act_fp4_dev: codes padded to whole
+ * 256-column stages and scale bytes in the scale-factor tile order of the block-scaled MMA, padding included, so
+ * the buffer needs no clearing.  The layout is internal (it depends on the token tile the matmul picks for M).
+ * razer_gemm_w4a4_fp4: razer_gemm_w4a4(use_native_fp4 = 1) on such an operand; bit-identical results.  Workspace:
+ * RAZER_OP_GEMM_W4A4 (zeroed once by razer_workspace_init). */
+int razer_fp4_act_bytes(int M, int K, size_t* bytes_out);
+int razer_quant_act_fp4(const void* x_dev, int M, int K, const float* tensor_scale_in_dev,
+                        uint32_t* amax_scratch_dev, void* act_fp4_dev, float* tensor_scale_out_dev,
+                        void* stream);
+int razer_gemm_w4a4_fp4(const razer_desc* d, const void* packed_w_dev, const void* act_fp4_dev,
+                        const float* act_tensor_scale_dev, int M, void* y_dev, void* workspace_dev,
+                        size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,7 @@ EXPORTS = (
     "razer_last_error", "razer_version", "razer_kernel_launches", "razer_packed_bytes", "razer_pack_layout", "razer_dequant",
     "razer_workspace_bytes", "razer_workspace_init", "razer_workspace_status", "razer_gemv", "razer_gemm", "razer_gemv_host", "razer_quant_act",
     "razer_decode_act", "razer_gemm_w4a4", "razer_gemv_static", "razer_quant_weight",
+    "razer_fp4_act_bytes", "razer_quant_act_fp4", "razer_gemm_w4a4_fp4",
 )
 
 
@@ -63,6 +64,10 @@ _lib.razer_quant_act.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p, c_vo
                                  c_void_p, c_void_p]
 _lib.razer_quant_weight.argtypes = [c_void_p, c_int, c_int, c_int, c_int, POINTER(c_float), c_int, c_void_p, c_void_p, c_void_p,
                                     c_void_p, c_void_p, c_void_p]
+_lib.razer_fp4_act_bytes.argtypes = [c_int, c_int, POINTER(c_size_t)]
+_lib.razer_quant_act_fp4.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+_lib.razer_gemm_w4a4_fp4.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_size_t,
+                                     c_void_p]
 _lib.razer_decode_act.argtypes = [c_void_p, c_void_p, c_int, c_int, c_float, c_void_p, c_void_p]
 _lib.razer_gemm_w4a4.argtypes = [POINTER(RazerDesc), c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_int,
                                  c_void_p, c_void_p, c_size_t, c_int, c_void_p]
@@ -229,6 +234,39 @@ def razer_quant_weight(w: torch.Tensor, sv_mag=(5.0, 8.0), remap_code: int = 0x8
     _check(_lib.razer_quant_weight(_ptr(w), N, K, int(block), int(bool(scale_aware)), mags, int(remap_code), _ptr(tensor_scale), _ptr(scratch),
                                    _ptr(codes), _ptr(scales), _ptr(out_scale), _stream()))
     return codes, scales, out_scale
+
+
+def razer_fp4_act_bytes(M: int, K: int) -> int:
+    n = c_size_t()
+    _check(_lib.razer_fp4_act_bytes(int(M), int(K), ctypes.byref(n)))
+    return n.value
+
+
+def razer_quant_act_fp4(x: torch.Tensor, tensor_scale: torch.Tensor | None = None, act_fp4: torch.Tensor | None = None,
+                        scratch: torch.Tensor | None = None):
+    """x bf16 [M, K] (device) -> (FP4 activation operand of the block-scaled kernel uint8 [bytes], tensor scale float32 [1])."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    M, K = x.shape
+    if act_fp4 is None:
+        act_fp4 = torch.empty(razer_fp4_act_bytes(M, K), dtype=torch.uint8, device=x.device)
+    out_scale = torch.empty(1, dtype=torch.float32, device=x.device)
+    if scratch is None:
+        scratch = _quant_act_scratch.get(x.device)
+        if scratch is None:
+            scratch = _quant_act_scratch[x.device] = torch.zeros(2, dtype=torch.int32, device=x.device)
+    _check(_lib.razer_quant_act_fp4(_ptr(x), M, K, _ptr(tensor_scale), _ptr(scratch), _ptr(act_fp4), _ptr(out_scale),
+                                    _stream()))
+    return act_fp4, out_scale
+
+
+def razer_gemm_w4a4_fp4(desc, packed, act_fp4, act_tensor_scale, M: int, y=None, workspace=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty((M, desc.N), dtype=torch.bfloat16, device=act_fp4.device)
+    if workspace is None:
+        workspace = alloc_workspace(desc, M, OP_GEMM_W4A4, act_fp4.device)
+    _check(_lib.razer_gemm_w4a4_fp4(ctypes.byref(desc), _ptr(packed), _ptr(act_fp4), _ptr(act_tensor_scale), int(M), _ptr(y),
+                                    _ptr(workspace), workspace.numel(), _stream()))
+    return y
 
 
 def razer_decode_act(codes: torch.Tensor, scales: torch.Tensor, sv_mag: float = 5.0) -> torch.Tensor:

@@ -76,6 +76,8 @@ size_t simt_workspace_bytes(const razer_desc*, int M);
 int launch_gemm_fp4(const razer_desc*, const void*, const uint8_t*, const uint8_t*, const float*, int, void*, void*, size_t,
                     cudaStream_t);
 size_t gemm_fp4_workspace_bytes(const razer_desc*, int M);
+int launch_gemm_fp4_prepared(const razer_desc*, const void*, const void*, const float*, int, void*, void*, size_t, cudaStream_t);
+int launch_quant_act_fp4(const void*, int, int, const float*, uint32_t*, void*, float*, cudaStream_t);
 int launch_gemm_umma(const razer_desc*, const void* packed, const void* x, int M, int ldx_K, float extra_scale,
                      const float* extra_scale_dev, void* y, void* ws, size_t ws_bytes, cudaStream_t);
 size_t umma_workspace_bytes(const razer_desc*, int M);
@@ -269,6 +271,39 @@ int razer_quant_act(const void* x_dev, int M, int K, float sv_mag, const float* 
   if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 8, "amax_scratch_dev"));
   return launch_quant_act(x_dev, M, K, sv_mag, tensor_scale_in_dev, amax_scratch_dev, act_codes_dev,
                           act_scales_dev, tensor_scale_out_dev, (cudaStream_t)stream);
+}
+
+int razer_fp4_act_bytes(int M, int K, size_t* bytes_out) {
+  if (!bytes_out) return set_error(RAZER_ERR_INVALID_ARG, "bytes_out is NULL");
+  if (M < 1 || K < 16 || K % 16) return set_error(RAZER_ERR_INVALID_ARG, "M=%d K=%d invalid (K %% 16 == 0)", M, K);
+  const Fp4ActLayout L = make_fp4_act_layout(M, K);
+  *bytes_out = L.codes_bytes + L.sfb_bytes;
+  return RAZER_OK;
+}
+
+int razer_quant_act_fp4(const void* x_dev, int M, int K, const float* tensor_scale_in_dev, uint32_t* amax_scratch_dev,
+                        void* act_fp4_dev, float* tensor_scale_out_dev, void* stream) {
+  if (M < 1 || K < 16 || K % 16) return set_error(RAZER_ERR_INVALID_ARG, "M=%d K=%d invalid (K %% 16 == 0)", M, K);
+  RAZER_TRY(check_ptr(x_dev, 16, "x_dev"));
+  RAZER_TRY(check_ptr(act_fp4_dev, 256, "act_fp4_dev"));
+  RAZER_TRY(check_ptr(tensor_scale_out_dev, 4, "tensor_scale_out_dev"));
+  if (!tensor_scale_in_dev) RAZER_TRY(check_ptr(amax_scratch_dev, 8, "amax_scratch_dev"));
+  return launch_quant_act_fp4(x_dev, M, K, tensor_scale_in_dev, amax_scratch_dev, act_fp4_dev, tensor_scale_out_dev,
+                              (cudaStream_t)stream);
+}
+
+int razer_gemm_w4a4_fp4(const razer_desc* d, const void* packed_w_dev, const void* act_fp4_dev,
+                        const float* act_tensor_scale_dev, int M, void* y_dev, void* workspace_dev, size_t workspace_bytes,
+                        void* stream) {
+  RAZER_TRY(check_desc(d));
+  if (M < 1) return set_error(RAZER_ERR_INVALID_ARG, "M=%d must be positive", M);
+  RAZER_TRY(check_ptr(packed_w_dev, 16, "packed_w_dev"));
+  RAZER_TRY(check_ptr(act_fp4_dev, 256, "act_fp4_dev"));
+  RAZER_TRY(check_ptr(act_tensor_scale_dev, 4, "act_tensor_scale_dev"));
+  RAZER_TRY(check_ptr(y_dev, 2, "y_dev"));
+  RAZER_TRY(check_ptr(workspace_dev, 256, "workspace_dev"));
+  return launch_gemm_fp4_prepared(d, packed_w_dev, act_fp4_dev, act_tensor_scale_dev, M, y_dev, workspace_dev,
+                                  workspace_bytes, (cudaStream_t)stream);
 }
 
 int razer_quant_weight(const float* w_dev, int N, int K, int block, int scale_aware, const float sv_mag[2], int remap_code,

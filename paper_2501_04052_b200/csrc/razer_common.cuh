@@ -76,6 +76,18 @@ __host__ __device__ inline Geometry make_geometry(int N, int K) {
 // Every matmul workspace starts with the device status word (0 = ok), on a block of its own.
 constexpr size_t WS_STATUS_BYTES = 256;
 
+// Layout of the FP4 activation operand as the block-scaled tensor-core kernel reads it (written by the activation
+// re-layout kernel or directly by the quantizer): codes [M][KP / 2] bytes (KP = K rounded up to whole 256-column
+// stages, zero beyond K, the nibbles of every 32-bit word in the packed form's order), then scale-factor tiles
+// [128-token tile][stage][chunk][512 bytes] (word 4 * (t % 32) + t / 32 of a tile = the four 7-bit scale bytes of
+// token t of the tile for the chunk's four blocks; zero for tokens beyond M and blocks beyond K).
+struct Fp4ActLayout {
+  int NT;            // tokens per tile of the matmul kernel: 128, or 256 above 128 tokens
+  int token_tiles, tiles128, spt, KP;
+  size_t codes_bytes, sfb_bytes;
+};
+Fp4ActLayout make_fp4_act_layout(int M, int K);   // host (razer_gemm_fp4.cu)
+
 // Decode parameters derived from a razer_desc on the host, passed to kernels by value.
 struct DecodeParams {
   float sv_mag[2];

@@ -576,31 +576,22 @@ __global__ void fp4_act_prep_kernel(const uint32_t* __restrict__ codes, const ui
 }
 
 struct Plan {
-  int NT, token_tiles, tiles128, steps_per_tile, grid, KP;
+  Fp4ActLayout act;
+  int grid;
   long long tiles, total_items;
-  size_t counters_bytes, slots_bytes, codes_bytes, sfb_bytes;
+  size_t counters_bytes, slots_bytes;
 };
 
 static Plan make_plan(const razer_desc* d, int M) {
   Plan p;
   const Geometry g = make_geometry(d->N, d->K);
-  p.NT = M > 128 ? 256 : 128;
-  if (const char* e = getenv("RAZER_FP4_NT")) {                       // tuning and test aid: force the token tile
-    const int v = atoi(e);
-    if (v == 128 || v == 256) p.NT = v;
-  }
-  p.token_tiles = (M + p.NT - 1) / p.NT;
-  p.tiles128 = p.token_tiles * (p.NT / 128);
-  p.steps_per_tile = (g.k_chunks + CH - 1) / CH;
-  p.KP = p.steps_per_tile * CH * CHUNK_K;
-  p.tiles = (long long)g.row_tiles * p.token_tiles;
-  p.total_items = p.tiles * p.steps_per_tile;
+  p.act = make_fp4_act_layout(M, d->K);
+  p.tiles = (long long)g.row_tiles * p.act.token_tiles;
+  p.total_items = p.tiles * p.act.spt;
   const int sms = sm_count();
   p.grid = (int)(p.total_items < sms ? p.total_items : sms);
   p.counters_bytes = align256((size_t)p.tiles * sizeof(uint32_t));
-  p.slots_bytes = (size_t)(p.grid > 148 ? p.grid : 148) * 2 * p.NT * TILE_ROWS * sizeof(float);
-  p.codes_bytes = align256((size_t)M * p.KP / 2);
-  p.sfb_bytes = (size_t)p.tiles128 * p.steps_per_tile * SF_BYTES;
+  p.slots_bytes = (size_t)(p.grid > 148 ? p.grid : 148) * 2 * p.act.NT * TILE_ROWS * sizeof(float);
   return p;
 }
 
@@ -642,17 +633,42 @@ static bool split_special_values(const float sv[2], uint32_t base[2], uint32_t r
 
 }  // namespace fp4_path
 
-size_t gemm_fp4_workspace_bytes(const razer_desc* d, int M) {
-  const fp4_path::Plan p = fp4_path::make_plan(d, M);
-  return WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes + p.codes_bytes + p.sfb_bytes;
+Fp4ActLayout make_fp4_act_layout(int M, int K) {
+  Fp4ActLayout L;
+  L.NT = M > 128 ? 256 : 128;
+  if (const char* e = getenv("RAZER_FP4_NT")) {                        // tuning and test aid: force the token tile
+    const int v = atoi(e);
+    if (v == 128 || v == 256) L.NT = v;
+  }
+  L.token_tiles = (M + L.NT - 1) / L.NT;
+  L.tiles128 = L.token_tiles * (L.NT / 128);
+  const int k_chunks = (K + CHUNK_K - 1) / CHUNK_K;
+  L.spt = (k_chunks + fp4_path::CH - 1) / fp4_path::CH;
+  L.KP = L.spt * fp4_path::CH * CHUNK_K;
+  L.codes_bytes = align256((size_t)M * L.KP / 2);
+  L.sfb_bytes = (size_t)L.tiles128 * L.spt * fp4_path::SF_BYTES;
+  return L;
 }
 
-int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_codes, const uint8_t* act_scales,
-                    const float* act_tensor_scale_dev, int M, void* y, void* ws, size_t ws_bytes, cudaStream_t st) {
+// workspace of the matmul proper: status word, tile counters, partial-tile slots
+size_t gemm_fp4_core_workspace_bytes(const razer_desc* d, int M) {
+  const fp4_path::Plan p = fp4_path::make_plan(d, M);
+  return WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes;
+}
+
+// ... plus the re-laid-out activation operand when the caller brings the interchange format
+size_t gemm_fp4_workspace_bytes(const razer_desc* d, int M) {
+  const fp4_path::Plan p = fp4_path::make_plan(d, M);
+  return WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes + p.act.codes_bytes + p.act.sfb_bytes;
+}
+
+// The matmul on a prepared activation operand (act_fp4: codes, then scale-factor tiles).
+int launch_gemm_fp4_prepared(const razer_desc* d, const void* packed, const void* act_fp4, const float* act_tensor_scale_dev,
+                             int M, void* y, void* ws, size_t ws_bytes, cudaStream_t st) {
   using namespace fp4_path;
   const Geometry g = make_geometry(d->N, d->K);
   const Plan p = make_plan(d, M);
-  const size_t need = gemm_fp4_workspace_bytes(d, M);
+  const size_t need = WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes;
   if (!ws || ws_bytes < need)
     return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
   Args a;
@@ -672,25 +688,24 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
   a.status = (uint32_t*)base_ws;
   a.counters = (uint32_t*)(base_ws + WS_STATUS_BYTES);
   a.slots = (float*)(base_ws + WS_STATUS_BYTES + p.counters_bytes);
-  uint8_t* codes_pad = (uint8_t*)(base_ws + WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes);
-  uint8_t* sfb = codes_pad + p.codes_bytes;
-  a.sfb = sfb;
+  uint8_t* codes_pad = (uint8_t*)const_cast<void*>(act_fp4);
+  a.sfb = codes_pad + p.act.codes_bytes;
   a.y = (__nv_bfloat16*)y;
   a.extra_scale = act_tensor_scale_dev;
   a.g = g;
   a.tensor_scale = d->tensor_scale;
   a.M = M;
-  a.token_tiles = p.token_tiles;
-  a.steps_per_tile = p.steps_per_tile;
+  a.token_tiles = p.act.token_tiles;
+  a.steps_per_tile = p.act.spt;
   a.total_items = p.total_items;
 
   const cuuint32_t estr[3] = {1, 1, 1};
   CUtensorMap tmap_x, tmap_w;
   {
     // padded activation codes as bytes: [M][KP / 2]; box = 128 bytes (one stage of k) x NT tokens
-    const cuuint64_t dims[2] = {(cuuint64_t)(p.KP / 2), (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)(p.KP / 2)};
-    const cuuint32_t box[2] = {128, (cuuint32_t)p.NT};
+    const cuuint64_t dims[2] = {(cuuint64_t)(p.act.KP / 2), (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)(p.act.KP / 2)};
+    const cuuint32_t box[2] = {128, (cuuint32_t)p.act.NT};
     const CUresult r = enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, codes_pad, dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -709,21 +724,6 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  {
-    const long long work = (long long)M * (p.KP / 32) + (long long)p.tiles128 * p.steps_per_tile * CH * 128;
-    long long blocks = (work + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks);
-    cfg.blockDim = dim3(256);
-    cfg.stream = st;
-    cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, fp4_act_prep_kernel, (const uint32_t*)act_codes, act_scales, M, d->K, p.KP,
-                                             p.tiles128, p.steps_per_tile, (uint32_t*)codes_pad, (uint32_t*)sfb);
-    count_launches(1);
-    RAZER_TRY(check_cuda(e, "fp4_act_prep_kernel launch"));
-  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)p.grid);
   cfg.blockDim = dim3(THREADS);
@@ -731,7 +731,7 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
   cudaError_t e;
-  if (p.NT == 128) {
+  if (p.act.NT == 128) {
     static bool attr_set = false;
     if (!attr_set) {
       RAZER_TRY(check_cuda(cudaFuncSetAttribute(razer_fp4_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -752,6 +752,39 @@ int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_
   }
   count_launches(1);
   return check_cuda(e, "razer_fp4_kernel launch");
+}
+
+// Interchange-format activations: re-lay them out into the workspace (one small kernel), then the matmul.
+int launch_gemm_fp4(const razer_desc* d, const void* packed, const uint8_t* act_codes, const uint8_t* act_scales,
+                    const float* act_tensor_scale_dev, int M, void* y, void* ws, size_t ws_bytes, cudaStream_t st) {
+  using namespace fp4_path;
+  const Plan p = make_plan(d, M);
+  const size_t core = WS_STATUS_BYTES + p.counters_bytes + p.slots_bytes;
+  const size_t need = core + p.act.codes_bytes + p.act.sfb_bytes;
+  if (!ws || ws_bytes < need)
+    return set_error(RAZER_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+  uint8_t* codes_pad = (uint8_t*)ws + core;
+  uint8_t* sfb = codes_pad + p.act.codes_bytes;
+  static const bool pdl = [] { const char* e = getenv("RAZER_PDL"); return !(e && e[0] == '0'); }();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  {
+    const long long work = (long long)M * (p.act.KP / 32) + (long long)p.act.tiles128 * p.act.spt * CH * 128;
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, fp4_act_prep_kernel, (const uint32_t*)act_codes, act_scales, M, d->K,
+                                             p.act.KP, p.act.tiles128, p.act.spt, (uint32_t*)codes_pad, (uint32_t*)sfb);
+    count_launches(1);
+    RAZER_TRY(check_cuda(e, "fp4_act_prep_kernel launch"));
+  }
+  return launch_gemm_fp4_prepared(d, packed, codes_pad, act_tensor_scale_dev, M, y, ws, core, st);
 }
 
 }  // namespace razer

@@ -85,10 +85,18 @@ __device__ __forceinline__ void quant_act_block(const uint4 v0, const uint4 v1, 
 // computed (Eq. 1), the grid first takes the tensor maximum: every CTA folds its share into sync[0] and counts
 // itself in sync[1], and all of them meet there (the launch is cooperative, so every CTA is resident; the wait is
 // bounded all the same).  sync[] must be zero when the kernel starts; the last CTA to finish sets it back to zero.
+// Where the quantizer writes: the interchange format (prepared == 0), or the FP4 activation operand of the
+// block-scaled tensor-core kernel (Fp4ActLayout: codes padded to KP columns with each word's nibbles in the packed
+// order, scale bytes in scale-factor tile order; the padding is written as zeros by this kernel too).
+struct QuantActOut {
+  int prepared;
+  int M, k16, kp16, spt, m_pad;      // rows; 16-element blocks per row of the input / of the padded operand; stages; padded rows
+};
+
 __global__ void __launch_bounds__(256) quant_act_fused_kernel(const uint4* __restrict__ x, long long n_blocks, float sv_mag,
                                                              const float* __restrict__ scale_in, uint32_t* sync,
                                                              uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                                                             float* __restrict__ scale_out) {
+                                                             float* __restrict__ scale_out, const QuantActOut o) {
   __shared__ uint32_t warp_max[8];
   __shared__ uint32_t amax_shared;
   float d32;
@@ -138,12 +146,37 @@ __global__ void __launch_bounds__(256) quant_act_fused_kernel(const uint4* __res
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = d32;
   const float d32x6 = __fmul_rn(d32, 6.0f);
-  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_blocks;
-       t += (long long)gridDim.x * blockDim.x) {
-    uint32_t w0, w1, sbyte;
-    quant_act_block(x[2 * t], x[2 * t + 1], d32, d32x6, sv_mag, w0, w1, sbyte);
-    codes[t] = make_uint2(w0, w1);
-    scales[t] = (uint8_t)sbyte;
+  if (!o.prepared) {
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_blocks;
+         t += (long long)gridDim.x * blockDim.x) {
+      uint32_t w0, w1, sbyte;
+      quant_act_block(x[2 * t], x[2 * t + 1], d32, d32x6, sv_mag, w0, w1, sbyte);
+      codes[t] = make_uint2(w0, w1);
+      scales[t] = (uint8_t)sbyte;
+    }
+  } else {
+    // one thread per block of the PADDED operand: (row m, block kb); blocks beyond K and rows beyond M are zeros
+    auto shuffle = [](uint32_t w) -> uint32_t {                        // element j of the word: nibble j -> nibble j / 2 + 4 (j % 2)
+      uint32_t r = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) r |= ((w >> (4 * j)) & 0xFu) << (4 * ((j >> 1) + 4 * (j & 1)));
+      return r;
+    };
+    const long long n_virtual = (long long)o.m_pad * o.kp16;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n_virtual;
+         t += (long long)gridDim.x * blockDim.x) {
+      const int m = (int)(t / o.kp16), kb = (int)(t - (long long)m * o.kp16);
+      uint32_t w0 = 0, w1 = 0, sbyte = 0;
+      if (m < o.M && kb < o.k16) {
+        const long long src = (long long)m * o.k16 + kb;
+        quant_act_block(x[2 * src], x[2 * src + 1], d32, d32x6, sv_mag, w0, w1, sbyte);
+      }
+      if (m < o.M) codes[(long long)m * o.kp16 + kb] = make_uint2(shuffle(w0), shuffle(w1));
+      // scale-factor tile of (128-token tile, stage, chunk); inside it word 4 * (t % 32) + t / 32, byte = block of the chunk
+      const int tile = m >> 7, tm = m & 127, step = kb >> 4, c = (kb >> 2) & 3;
+      const size_t at = (((size_t)tile * o.spt + step) * 4 + c) * 512 + (size_t)((tm & 31) * 4 + (tm >> 5)) * 4 + (kb & 3);
+      scales[at] = (uint8_t)(sbyte & 0x7Fu);
+    }
   }
   if (!scale_in) {
     __syncthreads();
@@ -334,10 +367,10 @@ int launch_quant_weight(const float* w, int N, int K, int block, int scale_aware
   return check_cuda(cudaGetLastError(), "quant_weight_kernel launch");
 }
 
-int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* scale_in,
-                     uint32_t* sync_scratch, uint8_t* codes, uint8_t* scales, float* scale_out,
-                     cudaStream_t st) {
+static int launch_quant_act_any(const void* x, int M, int K, float sv_mag, const float* scale_in, uint32_t* sync_scratch,
+                                uint8_t* codes, uint8_t* scales, float* scale_out, const QuantActOut& o, cudaStream_t st) {
   const long long n_blocks = (long long)M * (K / 16);
+  const long long n_work = o.prepared ? (long long)o.m_pad * o.kp16 : n_blocks;
   const int threads = 256;
   static int max_ctas = 0;                                             // CTAs that are resident together (cooperative launch)
   if (!max_ctas) {
@@ -348,7 +381,7 @@ int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* sca
                          "cudaOccupancyMaxActiveBlocksPerMultiprocessor"));
     max_ctas = sms * (per_sm < 1 ? 1 : per_sm);
   }
-  long long b = (n_blocks + threads - 1) / threads;
+  long long b = (n_work + threads - 1) / threads;
   const int grid = (int)(b < 1 ? 1 : (b > max_ctas ? max_ctas : b));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
@@ -360,9 +393,31 @@ int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* sca
   cfg.attrs = attr;
   cfg.numAttrs = scale_in ? 0 : 1;                                     // the grid only meets when it computes the scale
   const cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_fused_kernel, (const uint4*)x, n_blocks, sv_mag, scale_in,
-                                           sync_scratch, (uint2*)codes, scales, scale_out);
+                                           sync_scratch, (uint2*)codes, scales, scale_out, o);
   count_launches(1);
   return check_cuda(e, "quant_act_fused_kernel launch");
+}
+
+int launch_quant_act(const void* x, int M, int K, float sv_mag, const float* scale_in,
+                     uint32_t* sync_scratch, uint8_t* codes, uint8_t* scales, float* scale_out,
+                     cudaStream_t st) {
+  QuantActOut o = {};
+  return launch_quant_act_any(x, M, K, sv_mag, scale_in, sync_scratch, codes, scales, scale_out, o, st);
+}
+
+// Plain NVFP4 quantization (no special value) straight into the FP4 activation operand of the block-scaled kernel.
+int launch_quant_act_fp4(const void* x, int M, int K, const float* scale_in, uint32_t* sync_scratch, void* act_fp4,
+                         float* scale_out, cudaStream_t st) {
+  const Fp4ActLayout L = make_fp4_act_layout(M, K);
+  QuantActOut o;
+  o.prepared = 1;
+  o.M = M;
+  o.k16 = K / 16;
+  o.kp16 = L.KP / 16;
+  o.spt = L.spt;
+  o.m_pad = L.tiles128 * 128;
+  uint8_t* codes = (uint8_t*)act_fp4;
+  return launch_quant_act_any(x, M, K, 0.0f, scale_in, sync_scratch, codes, codes + L.codes_bytes, scale_out, o, st);
 }
 
 }  // namespace razer

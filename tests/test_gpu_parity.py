@@ -395,6 +395,37 @@ def test_w4a4_native_fp4_forced_token_tile(b, monkeypatch, nt, M):
     _w4a4_native_check(b, desc, packed, wc, ws, wd, ac, as_, ats)
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 512, 8192), (17, 200, 464), (300, 260, 1040), (130, 390, 2320)])
+def test_w4a4_fp4_prepared_operand_matches_the_interchange_route(b, M, N, K):
+    """razer_quant_act_fp4 + razer_gemm_w4a4_fp4 (the quantizer writes the tensor core's operand layout itself)
+    against razer_quant_act(sv_mag = 0) + razer_gemm_w4a4(use_native_fp4): same tensor scale, bit-identical outputs,
+    and the outputs within the matmul bars of the oracle's W4A4 result.  The operand buffer starts as garbage: the
+    quantizer has to write its padding too."""
+    w = inputs.student_t_weights(N, K, 320 + M, outlier_frac=0.001).numpy()
+    wc, ws, wd = ro.quantize_weight(w)
+    desc = b.make_desc(N, K, float(wd))
+    packed = b.razer_pack_layout(desc, torch.from_numpy(wc).cuda(), torch.from_numpy(ws).cuda())
+    x = inputs.activations(M, K, 321, outlier_channel_frac=0.01).cuda()
+    ac, as_, ats = b.razer_quant_act(x, sv_mag=0.0)
+    wsb = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+    y_ref = b.razer_gemm_w4a4(desc, packed, ac, as_, ats, workspace=wsb, use_native_fp4=True).clone()
+    b.razer_workspace_status(wsb)
+    buf = torch.full((b.razer_fp4_act_bytes(M, K),), 0xA5, dtype=torch.uint8, device="cuda")
+    act, ats2 = b.razer_quant_act_fp4(x, act_fp4=buf)
+    assert ats2.item() == ats.item()
+    wsb2 = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+    y = b.razer_gemm_w4a4_fp4(desc, packed, act, ats2, M, workspace=wsb2)
+    b.razer_workspace_status(wsb2)
+    assert torch.equal(y, y_ref)
+    given = torch.tensor([0.01], dtype=torch.float32, device="cuda")          # a given tensor scale: no grid rendezvous
+    act3, ats3 = b.razer_quant_act_fp4(x, tensor_scale=given)
+    ac3, as3, _ = b.razer_quant_act(x, sv_mag=0.0, tensor_scale=given)
+    y3 = b.razer_gemm_w4a4_fp4(desc, packed, act3, ats3, M, workspace=wsb2)
+    y3_ref = b.razer_gemm_w4a4(desc, packed, ac3, as3, ats3, workspace=wsb, use_native_fp4=True)
+    assert torch.equal(y3, y3_ref)
+    _w4a4_native_check(b, desc, packed, wc, ws, wd, ac, as_, ats)
+
+
 def test_w4a4_native_fp4_decodes_bit_exactly(b):
     """One-hot NVFP4 activations (code 1.0, block scale 1.0) through the two-pass path: y[m, n] is the tensor
     scale times one decoded weight, exact whatever the accumulation order, so main + comp is checked bit for bit."""
