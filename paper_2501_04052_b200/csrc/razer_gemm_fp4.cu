@@ -13,7 +13,8 @@
 // when there are more than 128), both K-major FP4 in shared memory with the 128-byte swizzle (one row = 256
 // codes = one stage of four chunks).  Warp 0 = weight producer (TMA box of packed bytes into a ring of its own,
 // released by the remap warps as soon as they have read it), warp 1 = TMEM owner and MMA issuer, warps 2..17 =
-// remap (thread = weight row and half of a stage's chunks; two groups of eight warps take the stages in turn)
+// remap (thread = weight row and one of a stage's four chunks; all sixteen warps take every stage, alternating
+// between two operand slots so that one stage is remapped while the previous one is multiplied)
 // and epilogue, warp 18 = activation producer (codes by TMA, scale-factor tiles by bulk copy, into a ring
 // released by the MMAs' completion).  A remap thread reads its row's packed blocks, finds the special-value
 // nibbles (the only nibbles that are 0x0 in the packed form), builds the two code words with two integer
@@ -40,8 +41,8 @@ namespace fp4_path {
 
 constexpr int CH = 4;                                 // chunks per stage: 256 codes = one 128-byte swizzled row
 constexpr int WSTAGES = 4;                            // packed-weight ring (released by the remap warps)
-constexpr int ASTAGES = 2;                            // remapped-operand ring, one slot per remap group
-constexpr int NRW = 16;                               // remap warps: two groups of eight
+constexpr int ASTAGES = 2;                            // remapped-operand ring: one slot is remapped while the other is multiplied
+constexpr int NRW = 16;                               // remap warps: four per chunk of a stage
 constexpr int THREADS = 64 + 32 * NRW + 32;           // + W producer, MMA warp, X producer
 constexpr int W_BYTES = CH * CHUNK_BYTES;             // 18432 packed weight bytes of a stage
 constexpr int SF_TILE_BYTES = 512;                    // scale factors of 128 rows x one chunk
@@ -149,7 +150,7 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const uint32_t bar_wfull = smem_u32(bars);            // [WSTAGES] TMA -> remap
-  const uint32_t bar_wempty = bar_wfull + 8 * WSTAGES;  // [WSTAGES] remap group (256 threads) -> TMA
+  const uint32_t bar_wempty = bar_wfull + 8 * WSTAGES;  // [WSTAGES] remap warps -> TMA
   const uint32_t bar_xfull = bar_wempty + 8 * WSTAGES;  // [XSTAGES] TMA -> MMA
   const uint32_t bar_xempty = bar_xfull + 8 * XSTAGES;  // [XSTAGES] MMA commit -> TMA
   const uint32_t bar_afull = bar_xempty + 8 * XSTAGES;  // [ASTAGES] remap -> MMA
@@ -173,14 +174,14 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   if (threadIdx.x == 0) {
     for (int i = 0; i < WSTAGES; ++i) {
       mbar_init(bar_wfull + 8 * i, 1);
-      mbar_init(bar_wempty + 8 * i, 256);
+      mbar_init(bar_wempty + 8 * i, 32 * NRW);
     }
     for (int i = 0; i < XSTAGES; ++i) {
       mbar_init(bar_xfull + 8 * i, 1);
       mbar_init(bar_xempty + 8 * i, 1);
     }
     for (int i = 0; i < ASTAGES; ++i) {
-      mbar_init(bar_afull + 8 * i, 256);
+      mbar_init(bar_afull + 8 * i, 32 * NRW);
       mbar_init(bar_aempty + 8 * i, 1);
     }
     mbar_init(bar_accfull, 1);
@@ -327,12 +328,11 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // ===================== remap (thread = weight row) + epilogue =====================
     const int row = 32 * (warp & 3) + lane;              // weight row of the tile = TMEM lane of its outputs
     const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
-    // Eight warps remap one item together: warps w and w + 4 of a group own the same 32 rows (a warp reaches only
-    // the TMEM lanes 32 * (warp % 4) .. + 31, which the epilogue needs) and take two of the stage's four chunks each.
-    const int group = (warp - 2) >> 3;
-    const int half = ((warp - 2) >> 2) & 1;
-    constexpr int GROUPS = NRW / 8;
-    static_assert(GROUPS == ASTAGES && WSTAGES % GROUPS == 0, "an operand slot per group; a weight stage always serves the same group");
+    // All sixteen warps remap every item: warps w, w + 4, w + 8, w + 12 own the same 32 rows (a warp reaches only the
+    // TMEM lanes 32 * (warp % 4) .. + 31, which the epilogue needs) and take one of the stage's four chunks each.
+    // The item after it goes into the other operand slot, so its remap runs while this item's MMAs execute.
+    const int chunk = (warp - 2) >> 2;
+    static_assert(NRW == 4 * CH, "one set of four warps per chunk");
     constexpr int EPI_SETS = NRW / 4;                     // sets of four warps (all lane quarters) share the columns
     const int col_lo = 16 * ((((warp - 2) >> 2) * (NT / 16)) / EPI_SETS);
     const int col_hi = 16 * (((((warp - 2) >> 2) + 1) * (NT / 16)) / EPI_SETS);
@@ -361,23 +361,20 @@ razer_fp4_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t row_off = (uint32_t)row * 128;        // this row inside an operand tile
     const uint32_t sw7 = (uint32_t)row & 7u;              // 128-byte swizzle: 16-byte unit u of row r sits at u ^ (r % 8)
     const uint32_t sf_word = (uint32_t)((row & 31) * 4 + (row >> 5)) * 4;
-    int turn = 0;                                        // item i is remapped by group i % GROUPS
-    for (int i = 0; i < n_items; ++i, cur.next(spt), turn = (turn + 1 == GROUPS ? 0 : turn + 1)) {
+    for (int i = 0; i < n_items; ++i, cur.next(spt)) {
       const int tile = cur.tile, step = cur.step;
       const bool seg_last = (i + 1 == n_items) || step == spt - 1;
       const int nch = min(CH, a.g.k_chunks - step * CH);
-      if (turn == group) {
-        // The operand slot and (WSTAGES being a multiple of GROUPS) the weight stage always serve this group, so
-        // the group sees every phase of both barriers and its parity waits are sound.
+      {
+        // every remap thread sees every phase of the barriers it waits on, so the parity waits are sound
         if (!wait_all(bar_aempty + 8 * cur.as, (uint32_t)cur.aph ^ 1u, 26)) break;
         if (!wait_all(bar_wfull + 8 * cur.ws, (uint32_t)cur.wph, 25)) break;
         const uint32_t st = smem_addr(smem_w) + (uint32_t)cur.ws * W_BYTES + strip_off;
         const uint32_t am = smem_addr(smem_a) + (uint32_t)cur.as * ASTAGE_BYTES + row_off;
         const uint32_t ac = am + A_TILE_BYTES;
         const uint32_t sfa = smem_addr(smem_a) + (uint32_t)cur.as * ASTAGE_BYTES + 2 * A_TILE_BYTES + sf_word;
-#pragma unroll
-        for (int cc = 0; cc < CH / 2; ++cc) {
-          const int c = half * (CH / 2) + cc;
+        {
+          const int c = chunk;
           if (c < nch) {
             const uint32_t ck = st + c * PIECE_BYTES;
             const uint2 sq = lds64(ck + scale_off);
