@@ -509,6 +509,26 @@ def test_repeated_launches_are_bit_identical(b, M, N, K):
     assert rel_fro_bits(first[:, torch.from_numpy(rows).cuda()], ref) <= TOL
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 8192, 8192), (2048, 4096, 4096), (100, 11008, 4096)])
+def test_repeated_fp4_launches_are_bit_identical(b, M, N, K):
+    """The block-scaled FP4 matmul repeated many times on one workspace must return the same bits: three rings, two
+    producer warps, sixteen remap warps and partial tiles combined across CTAs leave room for a rare ordering fault."""
+    codes, scales = inputs.random_codes(N, K, seed=150)
+    desc, packed = _pack(b, codes.numpy(), scales.numpy(), 0.002)
+    x = inputs.activations(M, K, 151, outlier_channel_frac=0.01).cuda()
+    act, ats = b.razer_quant_act_fp4(x)
+    ws = b.alloc_workspace(desc, M, b.OP_GEMM_W4A4, "cuda")
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    b.razer_gemm_w4a4_fp4(desc, packed, act, ats, M, y=y, workspace=ws)
+    first = y.clone()
+    differing = 0
+    for _ in range(1000):
+        b.razer_gemm_w4a4_fp4(desc, packed, act, ats, M, y=y, workspace=ws)
+        differing += int(not torch.equal(y, first))
+    b.razer_workspace_status(ws)
+    assert differing == 0, f"{differing} of 1000 launches differ from the first"
+
+
 # ------------------------------------------------------------------ host-buffer entry point, errors
 
 @pytest.mark.parametrize("pinned", [True, False])
