@@ -19,6 +19,8 @@ What is here, with the passage each function follows:
   dequant_d1/_d2       the dequantization product Delta32 * Delta8 * Xbar (Sec. 3)
   matmul_w4a16/_w4a4   definition: FP64-accumulated product rounded once to bf16
   two_pass_split       App. D.3 (B_main / B_comp decomposition)
+  quantize_fp16_block / dequant_fp16_block   Sec. 4.3 (deployment variant: block 128, FP16 block scale whose sign
+                       bit and top exponent bit carry the metadata); oracle only, no CUDA counterpart
 
 Floating point: the encoder works in FP32 in the operation order stated in each
 docstring (numpy float32 ops are IEEE, one rounding per op, never fused); the
@@ -523,3 +525,88 @@ def two_pass_split(codes, scales, sv_mag=(5.0, 8.0), remap_code=0x8):
     main = np.where(is_sv, base, q)
     comp = np.where(is_sv, rem, 0.0)
     return main, comp, split
+
+
+# --------------------------------------------------------------------------
+# Deployment variant of the weight-only kernel (Sec. 4.3): block 128, FP16 block scale
+# --------------------------------------------------------------------------
+
+def quantize_fp16_block(w: np.ndarray, sv_mag=(5.0, 8.0), remap_code: int = 0x8, block: int = 128,
+                        return_debug: bool = False):
+    """Sec. 4.3: one FP16 scale per block of `block` weights; its sign bit (bit 15) and most
+    significant exponent bit (bit 14) are redundant (a scale is positive and, for weights,
+    far below 2) and carry the 2-bit metadata (bit 15 = sign of the special value, bit 14 =
+    which magnitude, as in the 8-bit format).  There is no tensor scale.
+
+    Steps (FP32 unless stated): bmax = max|w| of the block; s = fl16(bmax / 6) (round to
+    nearest even onto FP16, then clamped into [2^-24, 2 - 2^-10] so that bit 14 stays
+    clear and a non-empty block keeps a positive scale); xs = w / fl32(s); Eq. 6-7 over
+    the whole block exactly as `quantize` does (candidates in metadata order, FP32 error
+    sums in ascending element order, first minimum).  Returns (codes [R, C/2] uint8,
+    scales [R, C/block] uint16).
+    """
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    assert w.ndim == 2 and w.shape[1] % block == 0 and remap_code in (0x0, 0x8)
+    R, C = w.shape
+    nb = C // block
+    f32 = np.float32
+    wb = w.reshape(R, nb, block)
+    bmax = np.max(np.abs(wb), axis=2).astype(np.float32)
+    s16 = (bmax / f32(6.0)).astype(np.float32).astype(np.float16)
+    s16 = np.clip(s16, np.float16(2.0 ** -24), np.float16(2.0 - 2.0 ** -10)).astype(np.float16)
+    s16 = np.where(bmax == 0, np.float16(0), s16).astype(np.float16)
+    sval = s16.astype(np.float32)
+    safe = np.where(sval == 0, f32(1.0), sval)
+    xs = (wb / safe[:, :, None]).astype(np.float32)
+    xs = np.where(sval[:, :, None] == 0, f32(0.0), xs)
+    ridx = round_to_fp4(xs)
+    rval = (np.where(np.signbit(xs), -1.0, 1.0) * _FP4_MAGS[ridx]).astype(np.float32)
+    d_r = np.abs(xs - rval).astype(np.float32)
+    cands = sv_candidates(sv_mag, SCALE_E3M3_META2)
+    errs32 = np.empty((len(cands), R, nb), dtype=np.float32)
+    errs64 = np.empty((len(cands), R, nb), dtype=np.float64)
+    use_sv = np.empty((len(cands), R, nb, block), dtype=bool)
+    for ci, v in enumerate(cands):
+        take = np.abs(xs - f32(v)).astype(np.float32) < d_r
+        q = np.where(take, f32(v), rval).astype(np.float32)
+        diff = (q - xs).astype(np.float32)
+        sq = (diff * diff).astype(np.float32)
+        acc = np.zeros((R, nb), dtype=np.float32)
+        for j in range(block):
+            acc = (acc + sq[:, :, j]).astype(np.float32)
+        errs32[ci] = acc
+        d64 = q.astype(np.float64) - xs.astype(np.float64)
+        errs64[ci] = np.sum(d64 * d64, axis=2)
+        use_sv[ci] = take
+    meta = np.argmin(errs32, axis=0).astype(np.uint16)
+    take = np.take_along_axis(use_sv, meta[None, :, :, None].astype(np.int64), axis=0)[0]
+    other_zero = remap_code ^ 0x8
+    std = (ridx | (np.signbit(xs).astype(np.uint8) << 3)).astype(np.uint8)
+    std = np.where(ridx == 0, other_zero, std).astype(np.uint8)
+    code = np.where(take, np.uint8(remap_code), std).astype(np.uint8)
+    code = np.where((sval == 0)[:, :, None], np.uint8(other_zero), code).reshape(R, C)
+    packed = (code[:, 0::2] | (code[:, 1::2] << 4)).astype(np.uint8)
+    # metadata order +m0, +m1, -m0, -m1: sign = meta >> 1 -> bit 15, select = meta & 1 -> bit 14
+    sbits = s16.view(np.uint16) | ((meta >> 1) << 15) | ((meta & 1) << 14)
+    sbits = np.where(sval == 0, 0, sbits).astype(np.uint16)
+    if return_debug:
+        d0 = rval.astype(np.float64) - xs.astype(np.float64)
+        return packed, sbits, dict(xs=xs, errs64=errs64, err_fp4=np.sum(d0 * d0, axis=2), meta=meta,
+                                   near_tie=_near_ties(errs64))
+    return packed, sbits
+
+
+def dequant_fp16_block(codes, scales16, sv_mag=(5.0, 8.0), remap_code: int = 0x8, block: int = 128):
+    """Dequantized weights of the FP16-scale variant, FP64: fl16 scale (bits 13:0 of the stored
+    word, i.e. sign and top exponent bit cleared) x element value, the special value given
+    by bits 15 (sign) and 14 (magnitude select)."""
+    scales16 = np.asarray(scales16, dtype=np.uint16)
+    s = (scales16 & np.uint16(0x3FFF)).view(np.float16).astype(np.float64)
+    sign = np.where((scales16 >> 15) & 1, -1.0, 1.0)
+    mag = np.where((scales16 >> 14) & 1, float(sv_mag[1]), float(sv_mag[0]))
+    sv = np.repeat(sign * mag, block, axis=1)
+    c = unpack_codes(codes)
+    vals = np.array([fp4_value(k) for k in range(16)], dtype=np.float64)[c]
+    other_zero = remap_code ^ 0x8
+    q = np.where(c == remap_code, sv, np.where(c == other_zero, 0.0, vals))
+    return q * np.repeat(s, block, axis=1)

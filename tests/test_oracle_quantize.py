@@ -373,3 +373,58 @@ def test_plain_nvfp4_is_eq_1_to_3_alone():
     c3, s3, _ = ro.quantize(d2v, ro.SCALE_E4M3_META1, None, tensor_scale=d32)
     assert np.array_equal(c3, c) and np.array_equal(s3, s)
     assert np.linalg.norm(d2v - xf) / np.linalg.norm(xf) < 0.12
+
+
+# --------------------------------------------------------------------------
+# deployment variant of Sec. 4.3: block 128, FP16 block scale carrying the metadata (oracle only)
+# --------------------------------------------------------------------------
+
+def test_fp16_block_scale_variant_bits_and_exact_cases():
+    """Sec. 4.3: the FP16 scale's sign bit and most significant exponent bit hold the metadata.  A block that is an
+    FP16 scale times grid values (special value included) is reproduced exactly, for each of the four special values;
+    the stored scale always has bit 14 clear once the metadata is masked off."""
+    rng = np.random.default_rng(5)
+    grid = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float64)
+    rows = []
+    svs = [5.0, 4.5, -5.0, -4.5]                       # both magnitudes below 6, so that Eq. 2's scale lets them be hit
+    for v in svs:
+        q = rng.choice(grid, size=128) * rng.choice([-1.0, 1.0], size=128)
+        q[0] = 6.0 if v > 0 else -6.0                   # pins the scale: bmax / 6 = s exactly
+        q[1:9] = v                                     # eight special values: no other candidate can match
+        rows.append(q * 0.0123291015625)               # an FP16-representable scale (101 * 2^-13)
+    w = np.array(rows, dtype=np.float32)
+    codes, s16 = ro.quantize_fp16_block(w, sv_mag=(5.0, 4.5))
+    assert [int(v) for v in (s16[:, 0] >> 14) & 3] == [0, 1, 2, 3]          # [sign | select] = metadata order +m0 +m1 -m0 -m1
+    assert np.all((s16 & 0x3FFF).view(np.float16).astype(np.float64) == 0.0123291015625)
+    assert np.array_equal(ro.dequant_fp16_block(codes, s16, sv_mag=(5.0, 4.5)), w.astype(np.float64))
+    # random weights: metadata-free scale is a positive FP16 below 2, Eq. 6 invariant, idempotent re-quantization
+    w = _weights(64, 1024, 60)
+    codes, s16, dbg = ro.quantize_fp16_block(w, return_debug=True)
+    sval = (s16 & 0x3FFF).view(np.float16).astype(np.float64)
+    assert np.all((sval > 0) & (sval < 2)) and np.all(((s16 & 0x3FFF) >> 14) == 0)
+    assert np.all(dbg["errs64"].min(axis=0) <= dbg["err_fp4"] + 1e-12)
+    d = ro.dequant_fp16_block(codes, s16)
+    c2, s2 = ro.quantize_fp16_block(d.astype(np.float32))
+    assert np.array_equal(s2 & 0x3FFF, s16 & 0x3FFF)
+    assert np.allclose(ro.dequant_fp16_block(c2, s2), d, rtol=0, atol=0) or np.mean(c2 == codes) > 0.999
+    assert np.linalg.norm(d - w) / np.linalg.norm(w) < 0.15
+
+
+def test_fp16_block_scale_variant_brute_force_on_tiny_blocks():
+    """Eq. 6-7 by enumeration on blocks of two elements: the encoder's reconstruction error equals the minimum over
+    the four special values and all 256 code vectors at the block's FP16 scale."""
+    rng = np.random.default_rng(12)
+    w = (rng.standard_t(5, size=(40, 4)) * 0.02).astype(np.float32)
+    codes, s16 = ro.quantize_fp16_block(w, block=2)
+    got = ((ro.dequant_fp16_block(codes, s16, block=2) - w.astype(np.float64)) ** 2).reshape(40, 2, 2).sum(axis=2)
+    cands = ro.sv_candidates((5.0, 8.0), ro.SCALE_E3M3_META2)
+    sval = (s16 & 0x3FFF).view(np.float16).astype(np.float64)
+    wb = w.reshape(40, 2, 2).astype(np.float64)
+    for r in range(40):
+        for b in range(2):
+            best = np.inf
+            for v in cands:
+                vals = np.array([ro.fp4_value(k) if k != 8 else v for k in range(16)]) * sval[r, b]
+                e = (vals[:, None] - wb[r, b][None, :]) ** 2
+                best = min(best, e[:, 0].min() + e[:, 1].min())
+            assert got[r, b] <= best * (1 + 1e-4) + 1e-18
